@@ -1,0 +1,173 @@
+/*
+ * hkv.h — C ABI of the HybridKV decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * One autoregressive step of attention over a hybrid-compressed KV cache, and the compression that
+ * builds that cache (paper: Section 3.3 "Hybrid KV Cache Compression" and Appendix A "Details of
+ * Hybrid KV Cache Compression").
+ *
+ *   static  KV heads: text-prior static pruning — the cache keeps (i) the observation window,
+ *                     (ii) every text token before it, (iii) the Top-M visual tokens before it by
+ *                     the window score s_w; decode attends densely over that compacted cache.
+ *   dynamic KV heads: chunk-wise retrieval — the sequence is cut into fixed-size chunks, each
+ *                     represented by the mean of its keys; every decode step scores the query
+ *                     against the chunk means, takes the top-k chunks its budget allows and attends
+ *                     over the tokens of those chunks only.
+ *
+ * "Head" always means KV head; the G = n_q_heads / n_kv_heads query heads of a group share it.
+ *
+ * Conventions
+ *   - plain C linkage; no exception crosses the boundary; no global state; every call returns a
+ *     status.  Argument errors are found on the host before anything is launched.
+ *   - "dev" pointers are device (HBM) addresses on the current CUDA device, "host" pointers are
+ *     ordinary host memory.  bf16 tensors are passed as void*.
+ *   - the caller owns every device buffer, including cache_mem and workspace.  The library never
+ *     allocates or frees device memory.  The opaque handle owns host metadata only.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All device
+ *     work is enqueued on it; calls return without synchronising unless stated.
+ *   - dense tensors are row-major with the last index fastest.
+ */
+#ifndef HKV_H_
+#define HKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HKV_OK = 0,
+  HKV_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, bad index                         */
+  HKV_ERR_SHAPE = 2,       /* inconsistent geometry (lengths, window, heads)                   */
+  HKV_ERR_BUDGET = 3,      /* a budget < 1                                                     */
+  HKV_ERR_WORKSPACE = 4,   /* cache_mem / workspace too small or misaligned (256 B)            */
+  HKV_ERR_UNSUPPORTED = 5, /* geometry outside what the kernels are built for                  */
+  HKV_ERR_CUDA = 6,        /* a CUDA runtime call failed                                       */
+  HKV_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (see hkv_last_device_error)   */
+  HKV_ERR_INDEX = 8        /* a device-side index check failed                                 */
+} hkv_status;
+
+/* flags */
+#define HKV_CAUSAL_WINDOW 1u /* mask key j > position of the window row inside S_w (variant; the
+                                paper's equation has no mask)                                  */
+#define HKV_OUT_F32 2u       /* hkv_decode_attn writes float32 instead of bf16                 */
+
+/* Geometry of one layer's cache.  Supported: head_dim = 128, 1 <= n_q_heads / n_kv_heads <= 16,
+ * chunk_size >= 1, 1 <= obs_window <= every seq_len. */
+typedef struct {
+  int32_t batch;         /* B                                                                  */
+  int32_t n_q_heads;     /* Hq                                                                 */
+  int32_t n_kv_heads;    /* Hkv                                                                */
+  int32_t head_dim;      /* d                                                                  */
+  int32_t max_seq_len;   /* C_max: row pitch of k, v, is_text, token_scores                    */
+  int32_t chunk_size;    /* cs: tokens per chunk of a dynamic head (Appendix A)                */
+  int32_t obs_window;    /* w: length of the observation window (Appendix A)                   */
+  float softmax_scale;   /* 0 -> 1/sqrt(head_dim); used by S_w and by decode attention         */
+  uint32_t flags;
+} hkv_config;
+
+typedef struct hkv_cache hkv_cache; /* opaque; host metadata of one layer's compressed cache */
+
+typedef struct {
+  int64_t retained_tokens;       /* sum over heads of tokens attended per step (upper bound for
+                                    dynamic heads: k * cs)                                     */
+  int64_t kv_bytes_resident;     /* bytes of K/V planes held in cache_mem                      */
+  int64_t summary_bytes;         /* bytes of chunk means held in cache_mem                     */
+  int64_t algorithmic_bytes_per_step; /* 512 B per retained token + 256 B per chunk mean read  */
+  int64_t cache_bytes;           /* bytes of cache_mem in use                                  */
+  int64_t workspace_bytes;       /* bytes of compress workspace required                       */
+  int32_t n_static, n_dynamic;   /* (b, h) units of each type                                  */
+  int32_t n_splits;              /* CTAs of the flash-decode launch                            */
+  int32_t launches_per_decode;   /* kernels one hkv_decode_attn enqueues                       */
+} hkv_stats;
+
+/* Sizes of the two caller-owned device buffers, from HOST inputs only (no device work, no sync).
+ * The keep-set of a static head always has min(budget, seq_len) tokens and a dynamic head always
+ * loads min(n_chunks, ceil(budget / cs)) chunks (Appendix A: "determined by the per-head budget and
+ * chunk size"), so no size depends on device data.
+ *   seq_lens  host int32 [B]        token count C_b of each sequence, 1 <= C_b <= max_seq_len
+ *   head_type host uint8 [B, Hkv]   0 = static, 1 = dynamic (Section 3.1's classification result)
+ *   budgets   host int32 [B, Hkv]   per-head token budget (Section 3.2's allocation result), >= 1;
+ *                                   values above C_b are clamped to C_b
+ * Out: bytes for cache_mem (lives as long as the cache) and for workspace (needed only until the
+ * work hkv_compress enqueued has finished). */
+hkv_status hkv_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type,
+                    const int32_t* budgets, size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Build one layer's compressed cache (Appendix A, both paragraphs).
+ *   k, v         dev bf16 [B, Hkv, C_max, d]   full prefill keys / values (read only)
+ *   q_obs        dev bf16 [B, w, Hq, d]        queries of the last w prompt tokens of each sequence
+ *                                              (Q[C-w:C] of Appendix A's S_w); may be NULL iff
+ *                                              token_scores is given
+ *   token_scores dev f32  [B, Hkv, C_max]      optional: replaces s_w for static heads
+ *   is_text      dev u8   [B, C_max]           1 = text token, 0 = visual token
+ *   seq_lens, head_type, budgets               host arrays as in hkv_plan
+ *   cache_mem    dev, >= cache_bytes, 256-B aligned; owned by the caller, must outlive the handle's
+ *                use; holds the compacted static K/V, the dynamic K/V and chunk means, index lists
+ *                and the decode scratch
+ *   workspace    dev, >= workspace_bytes, 256-B aligned; may be released once the stream has
+ *                passed the work of this call
+ * Static head: s_w = mean over the w*G window rows of softmax(q k^T * scale) over all C_b tokens;
+ * keep = window U text-before-window U Top-M visual-before-window (M = budget - w - #text), ties to
+ * the lower position; if the budget cannot hold window + text, text is ranked by s_w for the
+ * budget - w places left; if budget <= w the last `budget` tokens are kept.
+ * Dynamic head: chunk mean = float32 sum of the chunk's keys in token order / chunk length, rounded
+ * to nearest-even bf16; the last chunk may be shorter.
+ * k, v, q_obs, token_scores and is_text may be released once the stream has passed this call.
+ * On success *out receives a handle to free with hkv_cache_destroy. */
+hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                        const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                        const uint8_t* head_type, const int32_t* budgets, void* cache_mem,
+                        size_t cache_bytes, void* workspace, size_t workspace_bytes, void* stream,
+                        hkv_cache** out);
+
+/* One decode step over the compressed cache (Appendix A: score chunks by the inner product of the
+ * query with the chunk metadata, take the top chunks, attend together with the static cache).
+ *   q    dev bf16 [B, Hq, d]   the step's query
+ *   out  dev bf16 [B, Hq, d]   (float32 if HKV_OUT_F32) attention output
+ * Dynamic head: score_c = sum over the group's query heads of <q_g, mean_c> (float32), top-k with
+ * ties to the lower chunk id, softmax attention over the tokens of the selected chunks.  Static
+ * head: softmax attention over its kept tokens.  Heads are independent.  Allocates nothing, never
+ * synchronises, results are deterministic.  Calls on the same cache must not overlap on the GPU
+ * (they share the cache's scratch). */
+hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* stream);
+
+/* Decode several layers' caches with ONE launch sequence: queries q[i] / outputs out[i] belong to
+ * caches[i].  All caches must have been planned with the same geometry.  Benchmark aid for small
+ * per-layer work; a real model's layers are sequential.  host arrays of n pointers. */
+hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q, void* const* out,
+                                 int32_t n, void* stream);
+
+hkv_status hkv_cache_destroy(hkv_cache* cache);
+
+/* ---- introspection (parity tests, roofline numerator). These synchronise the given stream. ---- */
+
+/* kept positions of static head (b, h), ascending; host_out has room for `capacity` ints. */
+hkv_status hkv_get_static_indices(hkv_cache* cache, int32_t b, int32_t h, int32_t* host_out,
+                                  int32_t capacity, int32_t* n, void* stream);
+/* chunk ids the last hkv_decode_attn selected for dynamic head (b, h), ascending. */
+hkv_status hkv_get_selected_chunks(hkv_cache* cache, int32_t b, int32_t h, int32_t* host_out,
+                                   int32_t capacity, int32_t* n, void* stream);
+/* float32 chunk scores of the last hkv_decode_attn for dynamic head (b, h); n = n_chunks. */
+hkv_status hkv_get_chunk_scores(hkv_cache* cache, int32_t b, int32_t h, float* host_out,
+                                int32_t capacity, int32_t* n, void* stream);
+/* bf16 chunk means of dynamic head (b, h), [n_chunks, d] as uint16 bit patterns. */
+hkv_status hkv_get_summaries(hkv_cache* cache, int32_t b, int32_t h, uint16_t* host_out,
+                             int32_t capacity_rows, int32_t* n_chunks, void* stream);
+/* byte offset inside `workspace` of the float32 s_w [C_b] that hkv_compress computed for static
+ * head (b, h) (valid while the caller keeps the workspace). */
+hkv_status hkv_window_scores_offset(const hkv_cache* cache, int32_t b, int32_t h, size_t* offset);
+
+hkv_status hkv_cache_stats(const hkv_cache* cache, hkv_stats* stats);
+
+/* Device error word: code is HKV_OK, HKV_ERR_TIMEOUT or HKV_ERR_INDEX; detail identifies the place.
+ * Synchronises the stream. */
+hkv_status hkv_last_device_error(hkv_cache* cache, int32_t* code, int32_t* detail, void* stream);
+
+const char* hkv_status_string(hkv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HKV_H_ */

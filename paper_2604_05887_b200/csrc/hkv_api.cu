@@ -1,0 +1,386 @@
+// Host side of libhkv: argument checks, the planner (every size, offset and work list follows from
+// host inputs, so nothing here waits for the device) and the C ABI.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "hkv_internal.h"
+
+using namespace hkv;
+
+namespace {
+
+inline int64_t align_up(int64_t x, int64_t a = kAlign) { return (x + a - 1) / a * a; }
+
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      n <= 0) {
+    cudaGetLastError();   // clear
+    return 148;
+  }
+  return n;
+}
+
+hkv_status check_config(const hkv_config* cfg) {
+  if (!cfg) return HKV_ERR_INVALID_ARG;
+  if (cfg->batch < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->max_seq_len < 1) return HKV_ERR_SHAPE;
+  if (cfg->n_q_heads % cfg->n_kv_heads != 0) return HKV_ERR_SHAPE;
+  if (cfg->head_dim != kHeadDim) return HKV_ERR_UNSUPPORTED;
+  if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) return HKV_ERR_UNSUPPORTED;
+  if (cfg->chunk_size < 1 || cfg->obs_window < 1) return HKV_ERR_SHAPE;
+  if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32)) return HKV_ERR_INVALID_ARG;
+  if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return HKV_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads > 60000) return HKV_ERR_UNSUPPORTED;
+  return HKV_OK;
+}
+
+// Fills every host-side field of `c` (units, splits, header with offsets, sizes).
+hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type, const int32_t* budgets,
+                      hkv_cache& c, int64_t* ws_rowstat_off, int* n_col_tiles_max) {
+  hkv_status st = check_config(cfg);
+  if (st != HKV_OK) return st;
+  if (!seq_lens || !head_type || !budgets) return HKV_ERR_INVALID_ARG;
+  const int B = cfg->batch, Hkv = cfg->n_kv_heads, G = cfg->n_q_heads / Hkv, cs = cfg->chunk_size, w = cfg->obs_window;
+  for (int b = 0; b < B; ++b) {
+    if (seq_lens[b] < 1 || seq_lens[b] > cfg->max_seq_len) return HKV_ERR_SHAPE;
+    if (w > seq_lens[b]) return HKV_ERR_SHAPE;
+    for (int h = 0; h < Hkv; ++h) {
+      if (head_type[b * Hkv + h] > 1) return HKV_ERR_INVALID_ARG;
+      if (budgets[b * Hkv + h] < 1) return HKV_ERR_BUDGET;
+    }
+  }
+  c.cfg = *cfg;
+  c.units.clear();
+  c.splits.clear();
+  Header& H = c.hdr;
+  std::memset(&H, 0, sizeof(H));
+  H.batch = B; H.n_q_heads = cfg->n_q_heads; H.n_kv_heads = Hkv; H.group = G;
+  H.chunk_size = cs; H.obs_window = w; H.max_seq_len = cfg->max_seq_len; H.flags = cfg->flags;
+  H.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(cfg->head_dim));
+  H.n_units = B * Hkv;
+
+  int max_C = 0;
+  c.max_static_rows = c.max_dyn_rows = c.max_chunks = 0;
+  c.retained = c.kv_bytes = c.summary_bytes = c.algo_bytes = 0;
+  for (int b = 0; b < B; ++b) {
+    for (int h = 0; h < Hkv; ++h) {
+      Unit u;
+      std::memset(&u, 0, sizeof(u));
+      u.type = head_type[b * Hkv + h];
+      u.b = b; u.h = h; u.C = seq_lens[b];
+      u.budget = std::min(budgets[b * Hkv + h], u.C);
+      if (u.type == 0) {
+        u.n_tok = u.budget;
+        u.plane_rows = u.n_tok;
+        c.max_static_rows = std::max(c.max_static_rows, u.plane_rows);
+        max_C = std::max(max_C, u.C);
+        H.n_static++;
+        c.algo_bytes += 2ll * kRowBytes * u.n_tok;
+      } else {
+        u.n_chunks = (u.C + cs - 1) / cs;
+        u.k_sel = std::min(u.n_chunks, (u.budget + cs - 1) / cs);
+        const int64_t nt = static_cast<int64_t>(u.k_sel) * cs;
+        const int64_t pr = static_cast<int64_t>(u.n_chunks) * cs;
+        if (pr > 0x7FFFFFF0ll) return HKV_ERR_UNSUPPORTED;
+        u.n_tok = static_cast<int32_t>(nt);
+        u.plane_rows = static_cast<int32_t>(pr);
+        c.max_dyn_rows = std::max(c.max_dyn_rows, u.plane_rows);
+        c.max_chunks = std::max(c.max_chunks, u.n_chunks);
+        H.n_dynamic++;
+        c.algo_bytes += 2ll * kRowBytes * std::min<int64_t>(nt, u.C) + static_cast<int64_t>(kRowBytes) * u.n_chunks;
+        c.summary_bytes += static_cast<int64_t>(kRowBytes) * u.n_chunks;
+      }
+      c.retained += std::min(u.n_tok, u.C);
+      c.kv_bytes += 2ll * kRowBytes * u.plane_rows;
+      c.units.push_back(u);
+    }
+  }
+
+  // ---- splits: one wave of CTAs whenever the work allows it ----
+  const int target = sm_count();
+  int max_tiles = 1;
+  for (auto& u : c.units) max_tiles = std::max(max_tiles, (u.n_tok + kTile - 1) / kTile);
+  int tps = kDecWarps;
+  while (tps < max_tiles) {
+    int64_t n = 0;
+    for (auto& u : c.units) n += ((u.n_tok + kTile - 1) / kTile + tps - 1) / tps;
+    if (n <= target) break;
+    tps += kDecWarps;
+  }
+  int split_total = 0;
+  for (int pass = 0; pass < 2; ++pass) {     // static units first: their work does not wait for the selection
+    for (int i = 0; i < H.n_units; ++i) {
+      Unit& u = c.units[i];
+      if (u.type != pass) continue;
+      const int tiles = (u.n_tok + kTile - 1) / kTile;
+      u.n_splits = std::max(1, (tiles + tps - 1) / tps);
+      u.split_base = split_total;
+      for (int s = 0; s < u.n_splits; ++s) {
+        Split sp;
+        sp.unit = i; sp.tile_begin = s * tps; sp.tile_end = std::min(tiles, (s + 1) * tps); sp.slot = s;
+        c.splits.push_back(sp);
+      }
+      split_total += u.n_splits;
+    }
+  }
+  H.n_splits = split_total;
+
+  // ---- cache_mem layout ----
+  int64_t off = align_up(sizeof(Header));
+  H.units_off = off;     off = align_up(off + sizeof(Unit) * H.n_units);
+  H.splits_off = off;    off = align_up(off + sizeof(Split) * split_total);
+  H.dyn_list_off = off;  off = align_up(off + 4ll * std::max(1, H.n_dynamic));
+  H.sta_list_off = off;  off = align_up(off + 4ll * std::max(1, H.n_static));
+  const int64_t tables_end = off;
+  H.counters_off = off;  off = align_up(off + 4ll * H.n_units);
+  H.n_valid_off = off;   off = align_up(off + 4ll * H.n_units);
+  H.err_off = off;       off = align_up(off + 8);
+  H.partials_off = off;  off = align_up(off + 4ll * split_total * G * (kHeadDim + 2));
+  for (auto& u : c.units) {
+    u.idx_off = off;
+    off = align_up(off + 4ll * std::max(1, u.type == 0 ? u.n_tok : u.k_sel));
+    if (u.type == 1) {
+      u.scores_off = off;  off = align_up(off + 4ll * u.n_chunks);
+      u.summ_off = off;    off = align_up(off + static_cast<int64_t>(kRowBytes) * u.n_chunks);
+    }
+  }
+  for (auto& u : c.units) {
+    u.k_off = off;  off = align_up(off + static_cast<int64_t>(kRowBytes) * u.plane_rows);
+    u.v_off = off;  off = align_up(off + static_cast<int64_t>(kRowBytes) * u.plane_rows);
+  }
+  c.cache_bytes = static_cast<size_t>(off);
+  (void)tables_end;
+
+  // ---- workspace layout: s_w per static unit, then the row statistics of the window softmax ----
+  int64_t woff = 0;
+  for (auto& u : c.units) {
+    if (u.type == 0) { u.ws_scores_off = woff; woff = align_up(woff + 4ll * u.C); }
+  }
+  const int R = w * G, Rpad = (R + 15) / 16 * 16;
+  const int tiles_max = (max_C + 63) / 64;
+  if (ws_rowstat_off) *ws_rowstat_off = woff;
+  if (n_col_tiles_max) *n_col_tiles_max = tiles_max;
+  woff = align_up(woff + 8ll * H.n_static * tiles_max * Rpad + 8ll * H.n_static * Rpad);
+  c.workspace_bytes = static_cast<size_t>(std::max<int64_t>(woff, kAlign));
+  return HKV_OK;
+}
+
+bool bad_unit(const hkv_cache* c, int b, int h) {
+  return !c || b < 0 || h < 0 || b >= c->cfg.batch || h >= c->cfg.n_kv_heads;
+}
+
+hkv_status d2h(void* dst, const void* src, size_t bytes, cudaStream_t s) {
+  if (cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return HKV_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return HKV_ERR_CUDA;
+  return HKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+hkv_status hkv_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type, const int32_t* budgets,
+                    size_t* cache_bytes, size_t* workspace_bytes) {
+  if (!cache_bytes || !workspace_bytes) return HKV_ERR_INVALID_ARG;
+  try {
+    hkv_cache tmp;
+    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, tmp, nullptr, nullptr);
+    if (st != HKV_OK) return st;
+    *cache_bytes = tmp.cache_bytes;
+    *workspace_bytes = tmp.workspace_bytes;
+    return HKV_OK;
+  } catch (...) {
+    return HKV_ERR_INVALID_ARG;
+  }
+}
+
+hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                        const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                        const uint8_t* head_type, const int32_t* budgets, void* cache_mem, size_t cache_bytes,
+                        void* workspace, size_t workspace_bytes, void* stream, hkv_cache** out) {
+  if (!out) return HKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!k || !v || !is_text || !cache_mem || !workspace) return HKV_ERR_INVALID_ARG;
+  hkv_cache* c = nullptr;
+  try {
+    c = new hkv_cache();
+    int64_t ws_rowstat_off = 0;
+    int tiles_max = 0;
+    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, *c, &ws_rowstat_off, &tiles_max);
+    if (st == HKV_OK && c->hdr.n_static > 0 && !q_obs && !token_scores) st = HKV_ERR_INVALID_ARG;
+    if (st == HKV_OK && (cache_bytes < c->cache_bytes || workspace_bytes < c->workspace_bytes)) st = HKV_ERR_WORKSPACE;
+    if (st == HKV_OK && ((reinterpret_cast<uintptr_t>(cache_mem) | reinterpret_cast<uintptr_t>(workspace)) & (kAlign - 1)))
+      st = HKV_ERR_WORKSPACE;
+    if (st != HKV_OK) { delete c; return st; }
+    c->dev_base = static_cast<char*>(cache_mem);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const Header& H = c->hdr;
+
+    // tables: one host image, one copy
+    const size_t tables = static_cast<size_t>(H.counters_off);
+    std::vector<char> img(tables, 0);
+    std::memcpy(img.data(), &H, sizeof(H));
+    std::memcpy(img.data() + H.units_off, c->units.data(), sizeof(Unit) * c->units.size());
+    std::memcpy(img.data() + H.splits_off, c->splits.data(), sizeof(Split) * c->splits.size());
+    int32_t* dl = reinterpret_cast<int32_t*>(img.data() + H.dyn_list_off);
+    int32_t* sl = reinterpret_cast<int32_t*>(img.data() + H.sta_list_off);
+    for (int i = 0; i < H.n_units; ++i) {
+      if (c->units[i].type) *dl++ = i; else *sl++ = i;
+    }
+    bool ok = cudaMemcpyAsync(c->dev_base, img.data(), tables, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    // counters, n_valid, error word start at zero
+    ok = ok && cudaMemsetAsync(c->dev_base + H.counters_off, 0, static_cast<size_t>(H.partials_off - H.counters_off), s) ==
+                   cudaSuccess;
+    if (ok && H.n_static > 0) {
+      if (!token_scores)
+        ok = launch_window_scores(c->dev_base, static_cast<char*>(workspace), k, q_obs, H, c->units, ws_rowstat_off,
+                                  tiles_max, s) == cudaSuccess;
+      ok = ok && launch_static_select(c->dev_base, static_cast<char*>(workspace), token_scores, is_text, H, s) == cudaSuccess;
+      ok = ok && launch_gather_static(c->dev_base, k, v, H, c->max_static_rows, s) == cudaSuccess;
+    }
+    if (ok && H.n_dynamic > 0)
+      ok = launch_build_dynamic(c->dev_base, k, v, H, c->max_dyn_rows, c->max_chunks, s) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); delete c; return HKV_ERR_CUDA; }
+    *out = c;
+    return HKV_OK;
+  } catch (...) {
+    delete c;
+    return HKV_ERR_INVALID_ARG;
+  }
+}
+
+hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
+                                 void* stream) {
+  if (!caches || !q || !out || n < 1 || n > kMaxMulti) return HKV_ERR_INVALID_ARG;
+  DecodeBatch batch;
+  std::memset(&batch, 0, sizeof(batch));
+  batch.n = n;
+  for (int i = 0; i < n; ++i) {
+    const hkv_cache* c = caches[i];
+    if (!c || !q[i] || !out[i]) return HKV_ERR_INVALID_ARG;
+    if (c->hdr.group != caches[0]->hdr.group || ((c->hdr.flags ^ caches[0]->hdr.flags) & HKV_OUT_F32)) return HKV_ERR_SHAPE;
+    batch.cache[i] = c->dev_base;
+    batch.q[i] = q[i];
+    batch.out[i] = out[i];
+    batch.split_prefix[i + 1] = batch.split_prefix[i] + c->hdr.n_splits;
+    batch.dyn_prefix[i + 1] = batch.dyn_prefix[i] + c->hdr.n_dynamic;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (launch_select_chunks(batch, batch.dyn_prefix[n], s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  if (launch_flash_decode(batch, batch.split_prefix[n], caches[0]->hdr.group, (caches[0]->hdr.flags & HKV_OUT_F32) != 0, s) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return HKV_ERR_CUDA;
+  }
+  return HKV_OK;
+}
+
+hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* stream) {
+  if (!cache) return HKV_ERR_INVALID_ARG;
+  hkv_cache* one[1] = {cache};
+  const void* qs[1] = {q};
+  void* os[1] = {out};
+  return hkv_decode_attn_multi(one, qs, os, 1, stream);
+}
+
+hkv_status hkv_cache_destroy(hkv_cache* cache) {
+  delete cache;
+  return HKV_OK;
+}
+
+hkv_status hkv_get_static_indices(hkv_cache* c, int32_t b, int32_t h, int32_t* host_out, int32_t capacity, int32_t* n,
+                                  void* stream) {
+  if (bad_unit(c, b, h) || !host_out || !n) return HKV_ERR_INVALID_ARG;
+  const Unit& u = c->units[b * c->cfg.n_kv_heads + h];
+  if (u.type != 0) return HKV_ERR_INVALID_ARG;
+  *n = u.n_tok;
+  if (capacity < u.n_tok) return HKV_ERR_WORKSPACE;
+  return d2h(host_out, c->dev_base + u.idx_off, 4ull * u.n_tok, static_cast<cudaStream_t>(stream));
+}
+
+hkv_status hkv_get_selected_chunks(hkv_cache* c, int32_t b, int32_t h, int32_t* host_out, int32_t capacity, int32_t* n,
+                                   void* stream) {
+  if (bad_unit(c, b, h) || !host_out || !n) return HKV_ERR_INVALID_ARG;
+  const Unit& u = c->units[b * c->cfg.n_kv_heads + h];
+  if (u.type != 1) return HKV_ERR_INVALID_ARG;
+  *n = u.k_sel;
+  if (capacity < u.k_sel) return HKV_ERR_WORKSPACE;
+  return d2h(host_out, c->dev_base + u.idx_off, 4ull * u.k_sel, static_cast<cudaStream_t>(stream));
+}
+
+hkv_status hkv_get_chunk_scores(hkv_cache* c, int32_t b, int32_t h, float* host_out, int32_t capacity, int32_t* n,
+                                void* stream) {
+  if (bad_unit(c, b, h) || !host_out || !n) return HKV_ERR_INVALID_ARG;
+  const Unit& u = c->units[b * c->cfg.n_kv_heads + h];
+  if (u.type != 1) return HKV_ERR_INVALID_ARG;
+  *n = u.n_chunks;
+  if (capacity < u.n_chunks) return HKV_ERR_WORKSPACE;
+  return d2h(host_out, c->dev_base + u.scores_off, 4ull * u.n_chunks, static_cast<cudaStream_t>(stream));
+}
+
+hkv_status hkv_get_summaries(hkv_cache* c, int32_t b, int32_t h, uint16_t* host_out, int32_t capacity_rows,
+                             int32_t* n_chunks, void* stream) {
+  if (bad_unit(c, b, h) || !host_out || !n_chunks) return HKV_ERR_INVALID_ARG;
+  const Unit& u = c->units[b * c->cfg.n_kv_heads + h];
+  if (u.type != 1) return HKV_ERR_INVALID_ARG;
+  *n_chunks = u.n_chunks;
+  if (capacity_rows < u.n_chunks) return HKV_ERR_WORKSPACE;
+  return d2h(host_out, c->dev_base + u.summ_off, static_cast<size_t>(kRowBytes) * u.n_chunks,
+             static_cast<cudaStream_t>(stream));
+}
+
+hkv_status hkv_window_scores_offset(const hkv_cache* c, int32_t b, int32_t h, size_t* offset) {
+  if (bad_unit(c, b, h) || !offset) return HKV_ERR_INVALID_ARG;
+  const Unit& u = c->units[b * c->cfg.n_kv_heads + h];
+  if (u.type != 0) return HKV_ERR_INVALID_ARG;
+  *offset = static_cast<size_t>(u.ws_scores_off);
+  return HKV_OK;
+}
+
+hkv_status hkv_cache_stats(const hkv_cache* c, hkv_stats* st) {
+  if (!c || !st) return HKV_ERR_INVALID_ARG;
+  std::memset(st, 0, sizeof(*st));
+  st->retained_tokens = c->retained;
+  st->kv_bytes_resident = c->kv_bytes;
+  st->summary_bytes = c->summary_bytes;
+  st->algorithmic_bytes_per_step = c->algo_bytes;
+  st->cache_bytes = static_cast<int64_t>(c->cache_bytes);
+  st->workspace_bytes = static_cast<int64_t>(c->workspace_bytes);
+  st->n_static = c->hdr.n_static;
+  st->n_dynamic = c->hdr.n_dynamic;
+  st->n_splits = c->hdr.n_splits;
+  st->launches_per_decode = 1 + (c->hdr.n_dynamic > 0 ? 1 : 0);
+  return HKV_OK;
+}
+
+hkv_status hkv_last_device_error(hkv_cache* c, int32_t* code, int32_t* detail, void* stream) {
+  if (!c || !code || !detail) return HKV_ERR_INVALID_ARG;
+  int32_t w[2] = {0, 0};
+  hkv_status st = d2h(w, c->dev_base + c->hdr.err_off, sizeof(w), static_cast<cudaStream_t>(stream));
+  if (st != HKV_OK) return st;
+  *code = w[0];
+  *detail = w[1];
+  return HKV_OK;
+}
+
+const char* hkv_status_string(hkv_status s) {
+  switch (s) {
+    case HKV_OK: return "ok";
+    case HKV_ERR_INVALID_ARG: return "invalid argument";
+    case HKV_ERR_SHAPE: return "inconsistent shape";
+    case HKV_ERR_BUDGET: return "budget below one token";
+    case HKV_ERR_WORKSPACE: return "buffer too small or misaligned";
+    case HKV_ERR_UNSUPPORTED: return "unsupported geometry";
+    case HKV_ERR_CUDA: return "CUDA runtime error";
+    case HKV_ERR_TIMEOUT: return "device-side wait ran out";
+    case HKV_ERR_INDEX: return "device-side index check failed";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

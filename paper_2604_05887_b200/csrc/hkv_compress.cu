@@ -1,0 +1,352 @@
+// Compression kernels (run once per prompt and layer): observation-window scores s_w for static
+// heads, the text-prior keep-set, the gather into the compacted static cache, and for dynamic heads
+// the chunk means plus the copy of K/V into the cache.  K/V rows are written with their sixteen
+// 16-byte pieces XOR-permuted by (row & 7), the layout the flash-decode kernel stages with plain
+// bulk copies and reads with bank-conflict-free ldmatrix.
+#include "hkv_device.cuh"
+#include "hkv_internal.h"
+
+namespace hkv {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kWsTile = 64;      // key columns per CTA of the window-score kernels
+constexpr int kWsWarps = 8;
+
+__device__ __forceinline__ const Unit* unit_of(const char* cache, const Header* hdr, bool dynamic, int ordinal,
+                                               int* uid_out) {
+  const int32_t* list = reinterpret_cast<const int32_t*>(cache + (dynamic ? hdr->dyn_list_off : hdr->sta_list_off));
+  const int uid = list[ordinal];
+  if (uid_out) *uid_out = uid;
+  return reinterpret_cast<const Unit*>(cache + hdr->units_off) + uid;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Window scores.  S_w = softmax over ALL tokens of the w*G window rows' logits, s_w = mean of rows.
+// MODE 0: per (row, column tile) running max and exp-sum.  MODE 1: with the rows' final (max, sum)
+// known, column sums of the normalised probabilities -> s_w.
+// One CTA = one 64-token column tile of one static unit; warps loop over 16-row tiles of the
+// R = w*G rows; logits on tensor cores.
+// stats: float2 [n_static][n_tiles_max][Rpad], final: float2 [n_static][Rpad]
+// ---------------------------------------------------------------------------------------------
+template <int MODE>
+__global__ void __launch_bounds__(kWsWarps * 32)
+    window_scores_kernel(const char* cache, char* workspace, const __nv_bfloat16* kin, const __nv_bfloat16* q_obs,
+                         float2* stats, const float2* final_stats, int n_tiles_max, int Rpad) {
+  __shared__ __align__(128) uint8_t ktile[kWsTile * kRowBytes];
+  __shared__ float colsum[kWsWarps][kWsTile];
+
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  const Unit* u = unit_of(cache, hdr, false, blockIdx.y, nullptr);
+  const int C = u->C, j0 = blockIdx.x * kWsTile;
+  if (j0 >= C) return;
+  const int G = hdr->group, w = hdr->obs_window, Hq = hdr->n_q_heads, Hkv = hdr->n_kv_heads;
+  const int R = w * G;
+  const bool causal = (hdr->flags & HKV_CAUSAL_WINDOW) != 0;
+  const float sc = hdr->scale * kLog2e;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+
+  // stage the key tile (rows past C are zero), 16-byte pieces permuted by row & 7
+  const uint4* ksrc = reinterpret_cast<const uint4*>(
+      kin + (static_cast<size_t>(u->b) * Hkv + u->h) * static_cast<size_t>(hdr->max_seq_len) * kHeadDim);
+  for (int idx = tid; idx < kWsTile * 16; idx += kWsWarps * 32) {
+    const int row = idx >> 4, c = idx & 15;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (j0 + row < C) v = ksrc[static_cast<size_t>(j0 + row) * 16 + c];
+    *reinterpret_cast<uint4*>(ktile + row * kRowBytes + ((c ^ (row & 7)) << 4)) = v;
+  }
+  __syncthreads();
+
+  const uint32_t kbase = smem_u32(ktile);
+  const int mj = lane >> 3, mi = lane & 7;
+  const int krow = mi + ((mj >> 1) << 3), kcsel = mj & 1;
+  float cacc[8][2];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) cacc[n][0] = cacc[n][1] = 0.f;
+
+  const int n_mt = (R + 15) / 16;
+  for (int mt = warp; mt < n_mt; mt += kWsWarps) {
+    const int r0 = mt * 16 + g, r1 = r0 + 8;
+    const int i0 = r0 / G, i1 = r1 / G;   // window row index of each mma row
+    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(
+        q_obs + ((static_cast<size_t>(u->b) * w + i0) * Hq + u->h * G + (r0 - i0 * G)) * kHeadDim);
+    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(
+        q_obs + ((static_cast<size_t>(u->b) * w + i1) * Hq + u->h * G + (r1 - i1 * G)) * kHeadDim);
+    uint32_t qa[8][4];
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      qa[kk][0] = (r0 < R) ? q0[kk * 8 + t] : 0u;
+      qa[kk][2] = (r0 < R) ? q0[kk * 8 + 4 + t] : 0u;
+      qa[kk][1] = (r1 < R) ? q1[kk * 8 + t] : 0u;
+      qa[kk][3] = (r1 < R) ? q1[kk * 8 + 4 + t] : 0u;
+    }
+    float s[8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < 4; ++sl) {
+      const int r = sl * 16 + krow;
+      const uint32_t rowaddr = kbase + r * kRowBytes;
+      const uint32_t key = r & 7;
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(b0, b1, b2, b3, rowaddr + (((2 * kk + kcsel) ^ key) << 4));
+        mma_bf16(s[2 * sl], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
+        mma_bf16(s[2 * sl + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+      }
+    }
+    // scale (base-2 logits) and mask: columns past C, and keys after the row's own position if causal
+    const int lim0 = causal ? (C - w + i0) : (C - 1), lim1 = causal ? (C - w + i1) : (C - 1);
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int j = j0 + n * 8 + 2 * t + e;
+        s[n][e] = (j < C && j <= lim0) ? s[n][e] * sc : -INFINITY;
+        s[n][2 + e] = (j < C && j <= lim1) ? s[n][2 + e] * sc : -INFINITY;
+      }
+    }
+    if (MODE == 0) {
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+        mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      float z0 = 0.f, z1 = 0.f;
+      if (mx0 > -INFINITY) {
+#pragma unroll
+        for (int n = 0; n < 8; ++n) z0 += exp2f(s[n][0] - mx0) + exp2f(s[n][1] - mx0);
+      }
+      if (mx1 > -INFINITY) {
+#pragma unroll
+        for (int n = 0; n < 8; ++n) z1 += exp2f(s[n][2] - mx1) + exp2f(s[n][3] - mx1);
+      }
+      z0 += __shfl_xor_sync(0xffffffffu, z0, 1);
+      z0 += __shfl_xor_sync(0xffffffffu, z0, 2);
+      z1 += __shfl_xor_sync(0xffffffffu, z1, 1);
+      z1 += __shfl_xor_sync(0xffffffffu, z1, 2);
+      if (t == 0) {
+        float2* dst = stats + (static_cast<size_t>(blockIdx.y) * n_tiles_max + blockIdx.x) * Rpad;
+        if (r0 < R) dst[r0] = make_float2(mx0, z0);
+        if (r1 < R) dst[r1] = make_float2(mx1, z1);
+      }
+    } else {
+      const float2* fin = final_stats + static_cast<size_t>(blockIdx.y) * Rpad;
+      const float2 f0 = (r0 < R) ? fin[r0] : make_float2(0.f, 1.f);
+      const float2 f1 = (r1 < R) ? fin[r1] : make_float2(0.f, 1.f);
+      const float inv0 = (r0 < R) ? 1.f / f0.y : 0.f, inv1 = (r1 < R) ? 1.f / f1.y : 0.f;
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+          cacc[n][e] += exp2f(s[n][e] - f0.x) * inv0 + exp2f(s[n][2 + e] - f1.x) * inv1;
+      }
+    }
+  }
+  if (MODE == 1) {
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float v = cacc[n][e];
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (g == 0) colsum[warp][n * 8 + 2 * t + e] = v;
+      }
+    }
+    __syncthreads();
+    if (tid < kWsTile && j0 + tid < C) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w2 = 0; w2 < kWsWarps; ++w2) tot += colsum[w2][tid];
+      float* sw = reinterpret_cast<float*>(workspace + u->ws_scores_off);
+      sw[j0 + tid] = tot / static_cast<float>(R);
+    }
+  }
+}
+
+__global__ void window_rowreduce_kernel(const char* cache, const float2* stats, float2* final_stats, int n_tiles_max,
+                                        int Rpad) {
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  const Unit* u = unit_of(cache, hdr, false, blockIdx.x, nullptr);
+  const int R = hdr->obs_window * hdr->group;
+  const int n_tiles = (u->C + kWsTile - 1) / kWsTile;
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const float2* st = stats + static_cast<size_t>(blockIdx.x) * n_tiles_max * Rpad + r;
+    float M = -INFINITY;
+    for (int jt = 0; jt < n_tiles; ++jt) M = fmaxf(M, st[static_cast<size_t>(jt) * Rpad].x);
+    float Z = 0.f;
+    for (int jt = 0; jt < n_tiles; ++jt) {
+      const float2 v = st[static_cast<size_t>(jt) * Rpad];
+      if (v.x > -INFINITY) Z += v.y * exp2f(v.x - M);
+    }
+    final_stats[static_cast<size_t>(blockIdx.x) * Rpad + r] = make_float2(M, Z);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Static keep-set: window U text-before-window U Top-M visual-before-window by score (ties to the
+// lower position); when window + text exceed the budget, text is ranked instead; when the budget
+// does not exceed the window, the last `budget` tokens.  One CTA per static unit, ascending output.
+// ---------------------------------------------------------------------------------------------
+constexpr int kKeepThreads = 1024;
+
+__global__ void __launch_bounds__(kKeepThreads)
+    static_select_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text) {
+  __shared__ int hist[256];
+  __shared__ int wsum[96];
+  __shared__ int bc[4];
+  __shared__ int s_ntext;
+
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  int uid;
+  const Unit* u = unit_of(cache, hdr, false, blockIdx.x, &uid);
+  const int C = u->C, w = hdr->obs_window, budget = u->n_tok;
+  const int tid = threadIdx.x;
+  const uint8_t* txt = is_text + static_cast<size_t>(u->b) * hdr->max_seq_len;
+  const float* scores = token_scores
+                            ? token_scores + (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * hdr->max_seq_len
+                            : reinterpret_cast<const float*>(workspace + u->ws_scores_off);
+  int32_t* out = reinterpret_cast<int32_t*>(cache + u->idx_off);
+  const int hist_end = C - w;   // tokens before the window
+
+  if (tid == 0) s_ntext = 0;
+  __syncthreads();
+  int cnt = 0;
+  for (int i = tid; i < hist_end; i += kKeepThreads) cnt += txt[i] != 0;
+  for (int off = 16; off >= 1; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+  if ((tid & 31) == 0 && cnt) atomicAdd(&s_ntext, cnt);
+  __syncthreads();
+  const int n_text = s_ntext;
+
+  int emitted;
+  if (budget <= w) {
+    const int start = C - budget;
+    emitted = block_select_emit(
+        C, 0, [](int) { return 0u; }, [&](int i) { return i >= start; }, out, hist, wsum, bc);
+  } else {
+    const int room = budget - w;
+    const bool rank_text = n_text >= room;       // window + text do not fit: rank the text tokens
+    const int k = rank_text ? room : room - n_text;
+    emitted = block_select_emit(
+        C, k,
+        [&](int i) {
+          if (i >= hist_end) return 0u;
+          const bool is_t = txt[i] != 0;
+          return (is_t == rank_text) ? float_key(scores[i]) : 0u;
+        },
+        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, out, hist, wsum, bc);
+  }
+  if (tid == 0) {
+    reinterpret_cast<int32_t*>(cache + hdr->n_valid_off)[uid] = emitted;
+    if (emitted != budget) {
+      int32_t* err = reinterpret_cast<int32_t*>(cache + hdr->err_off);
+      atomicCAS(&err[0], 0, HKV_ERR_INDEX);
+      err[1] = kErrIndex;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row movers.  One half-warp per row: 16 lanes x 16 bytes; lanes 0-15 move the K row, 16-31 the V
+// row.  Destination piece c of plane row i goes to position c ^ (i & 7).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+    gather_rows_kernel(char* cache, const uint4* kin, const uint4* vin, int dynamic) {
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  const Unit* u = unit_of(cache, hdr, dynamic != 0, blockIdx.y, nullptr);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = lane & 15;
+  const bool is_v = lane >= 16;
+  const int rows = u->plane_rows;
+  const int32_t* idx = reinterpret_cast<const int32_t*>(cache + u->idx_off);
+  const size_t plane_in = (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * static_cast<size_t>(hdr->max_seq_len);
+  uint4* dst_plane = reinterpret_cast<uint4*>(cache + (is_v ? u->v_off : u->k_off));
+  const uint4* src = is_v ? vin : kin;
+  for (int rr = 0; rr < 8; ++rr) {
+    const int i = blockIdx.x * 64 + warp * 8 + rr;
+    if (i >= rows) break;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (dynamic) {
+      if (i < u->C) val = src[(plane_in + i) * 16 + c];
+    } else {
+      val = src[(plane_in + idx[i]) * 16 + c];
+    }
+    dst_plane[static_cast<size_t>(i) * 16 + (c ^ (i & 7))] = val;
+  }
+}
+
+// Chunk means: thread = one channel; float32 running sum over the chunk's tokens in order, float32
+// division by the chunk's own length, round-to-nearest-even to bf16.
+__global__ void __launch_bounds__(kHeadDim) chunk_means_kernel(char* cache, const __nv_bfloat16* kin) {
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  const Unit* u = unit_of(cache, hdr, true, blockIdx.y, nullptr);
+  const int cs = hdr->chunk_size, C = u->C, d = threadIdx.x;
+  const __nv_bfloat16* kp =
+      kin + (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * static_cast<size_t>(hdr->max_seq_len) * kHeadDim;
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(cache + u->summ_off);
+  for (int cc = 0; cc < 8; ++cc) {
+    const int c = blockIdx.x * 8 + cc;
+    if (c >= u->n_chunks) break;
+    const int t0 = c * cs, t1 = min(t0 + cs, C);
+    float acc = 0.f;
+    for (int tk = t0; tk < t1; ++tk) acc = __fadd_rn(acc, __bfloat162float(kp[static_cast<size_t>(tk) * kHeadDim + d]));
+    out[static_cast<size_t>(c) * kHeadDim + d] = __float2bfloat16_rn(__fdiv_rn(acc, static_cast<float>(t1 - t0)));
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, const void* q_obs, const Header& hdr,
+                                 const std::vector<Unit>&, int64_t ws_rowstat_off, int n_col_tiles_max,
+                                 cudaStream_t stream) {
+  if (hdr.n_static == 0) return cudaSuccess;
+  const int R = hdr.obs_window * hdr.group;
+  const int Rpad = (R + 15) / 16 * 16;
+  float2* stats = reinterpret_cast<float2*>(workspace + ws_rowstat_off);
+  float2* fin = stats + static_cast<size_t>(hdr.n_static) * n_col_tiles_max * Rpad;
+  dim3 grid(n_col_tiles_max, hdr.n_static);
+  window_scores_kernel<0><<<grid, kWsWarps * 32, 0, stream>>>(
+      cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
+      n_col_tiles_max, Rpad);
+  window_rowreduce_kernel<<<hdr.n_static, 256, 0, stream>>>(cache, stats, fin, n_col_tiles_max, Rpad);
+  window_scores_kernel<1><<<grid, kWsWarps * 32, 0, stream>>>(
+      cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
+      n_col_tiles_max, Rpad);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_static_select(char* cache, char* workspace, const float* token_scores, const uint8_t* is_text,
+                                 const Header& hdr, cudaStream_t stream) {
+  if (hdr.n_static == 0) return cudaSuccess;
+  static_select_kernel<<<hdr.n_static, kKeepThreads, 0, stream>>>(cache, workspace, token_scores, is_text);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_static(char* cache, const void* k, const void* v, const Header& hdr, int max_rows,
+                                 cudaStream_t stream) {
+  if (hdr.n_static == 0 || max_rows <= 0) return cudaSuccess;
+  dim3 grid((max_rows + 63) / 64, hdr.n_static);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(cache, static_cast<const uint4*>(k), static_cast<const uint4*>(v), 0);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_build_dynamic(char* cache, const void* k, const void* v, const Header& hdr, int max_rows,
+                                 int max_chunks, cudaStream_t stream) {
+  if (hdr.n_dynamic == 0) return cudaSuccess;
+  dim3 grid((max_rows + 63) / 64, hdr.n_dynamic);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(cache, static_cast<const uint4*>(k), static_cast<const uint4*>(v), 1);
+  dim3 grid2((max_chunks + 7) / 8, hdr.n_dynamic);
+  chunk_means_kernel<<<grid2, kHeadDim, 0, stream>>>(cache, static_cast<const __nv_bfloat16*>(k));
+  return cudaGetLastError();
+}
+
+}  // namespace hkv

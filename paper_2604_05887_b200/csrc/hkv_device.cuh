@@ -1,0 +1,187 @@
+// Device-side helpers shared by the kernels of libhkv: PTX wrappers (mbarrier, bulk copy, ldmatrix,
+// mma), the order-preserving float key, and a block-wide exact top-k selection that emits ascending
+// indices.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace hkv {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- mbarrier + bulk async copy (TMA engine, 1-D, no multicast) ----
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait (about a second of SM clocks): returns false when the limit ran out; the caller
+// records an error and leaves instead of spinning for ever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long start = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u && clock64() - start > 2000000000ll) return false;
+  }
+}
+// global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// ---- tensor-core tile ops (warp-level mma on 16x8x16 bf16 tiles, fp32 accumulate) ----
+__device__ __forceinline__ void ldsm_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                              uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// ---- order-preserving key of a finite float: larger float <=> larger key; every key > 0 ----
+__device__ __forceinline__ uint32_t float_key(float f) {
+  f = f + 0.0f;   // -0 -> +0 so that equal floats have equal keys
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Block-wide exact selection.  Among the n items, every item with always(i) is emitted, and of the
+// items with key(i) != 0 ("candidates") the k with the largest keys are emitted, equal keys going
+// to the lower index.  Emission is in ascending index order into out[]; returns the number emitted
+// (valid in every thread).  Requires k <= number of candidates, blockDim.x a multiple of 32 and at
+// most 1024.  hist: 256 ints, wsum: 3*32 ints, bc: 4 ints of shared memory.
+// ---------------------------------------------------------------------------------------------
+template <class KeyFn, class AlwaysFn>
+__device__ int block_select_emit(int n, int k, KeyFn key, AlwaysFn always, int32_t* out, int* hist, int* wsum,
+                                 int* bc) {
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+  uint32_t prefix = 0, mask = 0;
+  int need = k;   // how many still to take among the keys matching the prefix
+  if (k > 0) {
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += nthr) hist[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < n; i += nthr) {
+        uint32_t kv = key(i);
+        if (kv != 0 && (kv & mask) == prefix) atomicAdd(&hist[(kv >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // lane L owns bins [8L, 8L+8); find the highest bin b with count(bins > b) < need <= count(bins >= b)
+        int loc[8], tot = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { loc[j] = hist[lane * 8 + j]; tot += loc[j]; }
+        int above = 0;   // total of lanes above this one
+        int run = tot;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          int v = __shfl_down_sync(0xffffffffu, run, off);
+          if (lane + off < 32) run += v;
+        }
+        above = run - tot;   // sum over lanes > lane
+        if (above < need && need <= above + tot) {
+          int acc = above;
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+            if (acc < need && need <= acc + loc[j]) { bc[0] = lane * 8 + j; bc[1] = need - acc; }
+            acc += loc[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix |= static_cast<uint32_t>(bc[0]) << shift;
+      mask |= 0xFFu << shift;
+      need = bc[1];
+      __syncthreads();
+    }
+  }
+  const uint32_t T = (k > 0) ? prefix : 0xFFFFFFFFu;
+  if (k <= 0) need = 0;
+  // ordered emission
+  int emitted = 0, eq_seen = 0;
+  for (int base = 0; base < n; base += nthr) {
+    const int i = base + tid;
+    bool gt = false, eq = false, alw = false;
+    if (i < n) {
+      uint32_t kv = key(i);
+      alw = always(i);
+      gt = (kv != 0) && (kv > T);
+      eq = (kv != 0) && (kv == T);
+    }
+    const uint32_t beq = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) wsum[warp] = __popc(beq);
+    __syncthreads();
+    int eq_before = eq_seen, eq_total = 0;
+    for (int w2 = 0; w2 < nwarp; ++w2) {
+      int c = wsum[w2];
+      if (w2 < warp) eq_before += c;
+      eq_total += c;
+    }
+    const int my_eq_rank = eq_before + __popc(beq & ((1u << lane) - 1u));
+    const bool sel = alw || gt || (eq && my_eq_rank < need);
+    const uint32_t bsel = __ballot_sync(0xffffffffu, sel);
+    if (lane == 0) wsum[32 + warp] = __popc(bsel);
+    __syncthreads();
+    int sel_before = emitted, sel_total = 0;
+    for (int w2 = 0; w2 < nwarp; ++w2) {
+      int c = wsum[32 + w2];
+      if (w2 < warp) sel_before += c;
+      sel_total += c;
+    }
+    if (sel) out[sel_before + __popc(bsel & ((1u << lane) - 1u))] = i;
+    emitted += sel_total;
+    eq_seen += eq_total;
+    __syncthreads();
+  }
+  return emitted;
+}
+
+}  // namespace hkv

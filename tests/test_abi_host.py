@@ -1,0 +1,90 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, plans sizes, and rejects bad arguments before any launch."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def hkv():
+    from paper_2604_05887_b200.build import build_library
+    build_library()
+    from paper_2604_05887_b200 import binding
+    return binding
+
+
+def test_every_declared_symbol_is_exported(hkv):
+    header = open(os.path.join(ROOT, "include", "hkv.h")).read()
+    declared = set(re.findall(r"\b(hkv_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(hkv.EXPORTS)
+    for name in declared:
+        assert hasattr(hkv.lib, name), name
+
+
+def test_status_strings(hkv):
+    assert hkv.status_string(0) == "ok"
+    assert len({hkv.status_string(i) for i in range(9)}) == 9
+
+
+def _cfg(hkv, **kw):
+    base = dict(batch=2, n_q_heads=28, n_kv_heads=4, head_dim=128, max_seq_len=1000, chunk_size=32, obs_window=32)
+    base.update(kw)
+    return hkv.make_config(**base)
+
+
+def test_plan_sizes_grow_with_budget_and_are_aligned(hkv):
+    sl, ht = [1000, 900], [[0, 1, 0, 1]] * 2
+    c1, w1 = hkv.hkv_plan(_cfg(hkv), sl, ht, np.full((2, 4), 100))
+    c2, w2 = hkv.hkv_plan(_cfg(hkv), sl, ht, np.full((2, 4), 500))
+    assert c1 % 256 == 0 and w1 % 256 == 0 and c2 > c1 and w1 == w2
+    # dynamic heads keep the whole K/V resident: at least 2 * 256 B per token
+    assert c1 > 2 * 2 * 256 * 900
+
+
+@pytest.mark.parametrize("kw,sl,ht,bu,status", [
+    (dict(head_dim=64), [1000, 900], 0, 100, 5),
+    (dict(n_q_heads=30), [1000, 900], 0, 100, 2),
+    (dict(n_q_heads=68, n_kv_heads=4), [1000, 900], 0, 100, 5),
+    (dict(), [1001, 900], 0, 100, 2),
+    (dict(), [1000, 0], 0, 100, 2),
+    (dict(obs_window=901), [1000, 900], 0, 100, 2),
+    (dict(), [1000, 900], 2, 100, 1),
+    (dict(), [1000, 900], 0, 0, 3),
+    (dict(chunk_size=0), [1000, 900], 0, 100, 2),
+    (dict(flags=64), [1000, 900], 0, 100, 1),
+])
+def test_plan_rejects_bad_arguments(hkv, kw, sl, ht, bu, status):
+    with pytest.raises(hkv.HkvError) as e:
+        hkv.hkv_plan(_cfg(hkv, **kw), sl, np.full((2, 4), ht), np.full((2, 4), bu))
+    assert e.value.status == status
+
+
+def test_null_pointers_are_rejected(hkv):
+    import ctypes as C
+    cb, wb = C.c_size_t(0), C.c_size_t(0)
+    assert hkv.lib.hkv_plan(None, None, None, None, C.byref(cb), C.byref(wb)) == 1
+    assert hkv.lib.hkv_decode_attn(None, None, None, None) == 1
+    assert hkv.lib.hkv_cache_stats(None, None) == 1
+    h = C.c_void_p(None)
+    cfg = _cfg(hkv)
+    assert hkv.lib.hkv_compress(C.byref(cfg), None, None, None, None, None, None, None, None, None, 0, None, 0, None,
+                                C.byref(h)) == 1
+    assert h.value is None
+    assert hkv.lib.hkv_cache_destroy(None) == 0
+
+
+def test_split_plan_is_one_wave_for_bench_shape(hkv):
+    """cfg2-shaped layer: the flash-decode grid must not exceed one CTA per SM (148 without a device)."""
+    from paper_2604_05887_b200.binding import hkv_config
+    import ctypes as C
+    sl = [32768, 30000, 27000, 25000]
+    ht = np.array([[0, 1, 0, 0], [1, 0, 1, 0], [0, 0, 1, 1], [0, 1, 0, 0]])
+    bu = np.array([[int(np.ceil(0.1 * c))] * 4 for c in sl])
+    cfg = _cfg(hkv, batch=4, max_seq_len=32768, chunk_size=64)
+    cache_bytes, _ = hkv.hkv_plan(cfg, sl, ht, bu)
+    assert cache_bytes < 2 * 256 * 32768 * 16      # far below the full KV of the layer

@@ -1,0 +1,203 @@
+"""CUDA path vs CPU oracle, through the C ABI, on the same seeded inputs (needs a B200)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import hkv_inputs as hi
+from oracle import hkv_oracle as o
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    import parity_util
+    return parity_util
+
+
+def _geom(L, **kw):
+    for k, v in kw.items():
+        setattr(L, k, v)
+    return L
+
+
+def small(seed=5, B=2, C=700, cs=16, w=8, Hq=28, Hkv=4, budget=0.2, ragged=True, head_type=None, n_steps=2):
+    """cfg0-like values with free sizes (head_dim stays 128)."""
+    L = hi.tiny(seed=seed, B=B, C=C, chunk_size=cs, w=w, Hq=Hq, Hkv=Hkv, d=128, budget_fraction=budget,
+                n_steps=n_steps, ragged=ragged, head_type=head_type)
+    return L
+
+
+def test_cfg0_parity(P):
+    L = hi.cfg0(n_steps=3)
+    rep = P.compare_layer(L)
+    assert rep["stats"]["n_static"] == 2 and rep["stats"]["n_dynamic"] == 2
+    print("cfg0", rep)
+
+
+def test_cfg0_bf16_output(P):
+    L = hi.cfg0()
+    rep = P.compare_layer(L, flags=0)
+    print("cfg0 bf16 out", rep)
+
+
+@pytest.mark.parametrize("cs", [1, 7, 8, 16, 24, 32, 64, 128, 1000])
+def test_chunk_sizes(P, cs):
+    L = small(cs=cs, C=700, budget=0.23)
+    P.compare_layer(L)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 2), (28, 4), (16, 2), (24, 2), (16, 1)])
+def test_group_sizes(P, Hq, Hkv):
+    L = small(Hq=Hq, Hkv=Hkv, C=500, cs=16, B=2)
+    P.compare_layer(L)
+
+
+@pytest.mark.parametrize("budget_tokens", [1, 3, 8, 9, 40, 41, 300, 499, 500, 10 ** 6])
+def test_budget_edges(P, budget_tokens):
+    # window w = 8; #text before the window is ~ 30: covers budget < w, = w, window+text not fitting, full
+    L = small(C=500, cs=16, w=8, ragged=False, B=1, head_type=[[0, 1, 0, 1]])
+    L.budgets[:] = budget_tokens
+    rep = P.compare_layer(L)
+    if budget_tokens >= 500:
+        assert rep["stats"]["retained_tokens"] == 4 * 500
+
+
+def test_full_budget_matches_textbook_attention(P):
+    """100 % budget: both head types reduce to full-cache GQA attention (library routine)."""
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    L = small(C=1500, cs=32, B=2, head_type=[[0, 1, 1, 0], [1, 0, 0, 1]])
+    L.budgets[:] = L.seq_lens[:, None]
+    lc = LayerCache(L, flags=hkv.HKV_OUT_F32)
+    out = lc.decode(to_device_bf16(L.q[0])).cpu().numpy()
+    for b in range(L.batch):
+        C = int(L.seq_lens[b])
+        f = lambda u: torch.from_numpy(np.ascontiguousarray(u)).view(torch.bfloat16).to(torch.float64)
+        Q = f(L.q[0][b])[None, :, None, :]
+        K = f(L.k[b, :, :C]).repeat_interleave(L.group, dim=0)[None]
+        V = f(L.v[b, :, :C]).repeat_interleave(L.group, dim=0)[None]
+        ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V)[0, :, 0].numpy()
+        P.check_outputs(out[b], ref, "full budget")
+
+
+def test_token_scores_override(P):
+    L = small(C=600, cs=16, B=2)
+    rng = np.random.default_rng(9)
+    ts = rng.standard_normal((L.batch, L.n_kv_heads, L.max_seq_len)).astype(np.float32)
+    ts[0, :, 100:140] = 0.25          # a run of exact ties: the lower positions must win
+    ts[1, :, 7] = -0.0
+    ts[1, :, 9] = 0.0
+    P.compare_layer(L, token_scores=ts)
+
+
+def test_causal_window_variant(P):
+    from paper_2604_05887_b200 import binding as hkv
+    L = small(C=400, cs=16, w=16)
+    P.compare_layer(L, flags=hkv.HKV_OUT_F32 | hkv.HKV_CAUSAL_WINDOW)
+
+
+def test_custom_scale(P):
+    L = small(C=300, cs=8)
+    P.compare_layer(L, softmax_scale=0.05)
+
+
+def test_ragged_tail_chunk_and_many_splits(P):
+    L = small(C=5003, cs=32, B=3, budget=0.6, w=32)
+    rep = P.compare_layer(L)
+    assert rep["stats"]["n_splits"] > L.batch * L.n_kv_heads
+
+
+def test_determinism_and_static_independent_of_dynamic_budget():
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    L = small(C=3000, cs=32, B=2, head_type=[[0, 1, 1, 0], [1, 0, 0, 1]])
+    q = to_device_bf16(L.q[0])
+    outs = []
+    for rep in range(2):
+        lc = LayerCache(L)
+        a = lc.decode(q).clone()
+        b = lc.decode(q).clone()
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        outs.append(a)
+        lc.close()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+    L.budgets[L.head_type == 1] = 1700
+    lc = LayerCache(L)
+    c = lc.decode(q)
+    torch.cuda.synchronize()
+    G = L.group
+    for b in range(L.batch):
+        for h in range(L.n_kv_heads):
+            same = torch.equal(c[b, h * G:(h + 1) * G].view(torch.int16), outs[0][b, h * G:(h + 1) * G].view(torch.int16))
+            assert same == (L.head_type[b, h] == 0)
+
+
+def test_multi_layer_launch_equals_single_calls():
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    Ls = [hi.cfg1(layer=l, C=2048, block=256, n_steps=1) for l in range(3)]
+    lcs = [LayerCache(L) for L in Ls]
+    qs = [to_device_bf16(L.q[0]) for L in Ls]
+    single = [lc.decode(q).clone() for lc, q in zip(lcs, qs)]
+    outs = [lc.new_out() for lc in lcs]
+    hkv.hkv_decode_attn_multi([lc.handle for lc in lcs], qs, outs)
+    torch.cuda.synchronize()
+    for a, b in zip(single, outs):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_cfg1_layer(P):
+    L = hi.cfg1(layer=2, n_steps=2)
+    rep = P.compare_layer(L)
+    print("cfg1", rep)
+
+
+def test_cfg2_reduced(P):
+    L = hi.cfg2(layer=1, B=2, n_frames=12, min_frames=9)
+    rep = P.compare_layer(L)
+    print("cfg2 reduced", rep)
+
+
+def test_cfg3_reduced_planted_chunks(P):
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    L = hi.cfg3(layer=0, B=2, C=5000, block=512)
+    P.compare_layer(L)
+    lc = LayerCache(L)
+    lc.decode(to_device_bf16(L.q[0]))
+    for b in range(L.batch):
+        for h in range(L.n_kv_heads):
+            if L.head_type[b, h] == 1:
+                sel = hkv.hkv_get_selected_chunks(lc.handle, b, h)
+                assert set(L.planted[b, h].tolist()) <= set(sel.tolist())
+
+
+@pytest.mark.parametrize("budget,sf,cs", [(0.05, 0.5, 16), (0.2, 0.25, 128), (0.5, 0.75, 64), (1.0, 0.5, 32)])
+def test_cfg4_cells_reduced(P, budget, sf, cs):
+    L = hi.cfg4(budget, sf, cs, B=4, C=4096, block=512)
+    P.compare_layer(L)
+
+
+def test_cfg2_full_size_sampled_units(P):
+    """Bench configuration at full size (B=4, 32768 tokens, chunk 64): the launch shape bench.py times;
+    the oracle checks a sample of (b, h) units one by one."""
+    L = hi.cfg2(layer=0)
+    units = [(0, 0), (0, 3), (1, 1), (2, 2), (3, 0), (3, 3)]
+    rep = P.compare_layer(L, units=units)
+    print("cfg2 full", rep)
+
+
+def test_cfg3_full_length_sampled_units(P):
+    L = hi.cfg3(layer=0, B=2)
+    rep = P.compare_layer(L, units=[(0, 0), (0, 1), (1, 2), (1, 3)])
+    print("cfg3 50000", rep)
+
+
+def test_cfg4_full_size_cell_sampled(P):
+    L = hi.cfg4(0.10, 0.5, 32)
+    rep = P.compare_layer(L, units=[(0, 0), (5, 1), (9, 2), (15, 3)])
+    print("cfg4 cell", rep)
