@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the HybridKV decode hot path on B200.
+
+A *step* is one autoregressive decode step of attention over the hybrid-compressed KV cache of the
+whole model: one hkv_decode_attn per layer (chunk score + top-k for dynamic heads, split-K
+flash-decode over static and selected dynamic KV, merge), layers in sequence on one stream, captured
+once in a CUDA graph.  Default workload: the 28-layer, batch-4, 24K-32K-token video-like
+configuration ("cfg2": static fraction 0.6, budget 10 %, chunk 64) with seeded synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` = algorithmic HBM bytes per step (512 B per retained token
++ 256 B per chunk mean) summed over all ranks / step time; `us_per_step` is the step latency.
+Under torchrun every rank runs its own replica of the workload (different seed): weak scaling, no
+data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+NOMINAL_HBM_GBS = 8000.0           # the denominator the task statement names ("~8 TB/s")
+N_LAYERS = {"cfg0": 1, "cfg1": 28, "cfg2": 28, "cfg3": 28, "cfg4": 1}
+# DRAM bytes per launch of the flash-decode kernel from the ncu capture summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def layer_inputs(workload: str, layer: int, seed: int, threads: int):
+    import hkv_inputs as hi
+    if workload == "cfg0":
+        return hi.cfg0(seed=seed, layer=layer)
+    if workload == "cfg1":
+        return hi.cfg1(layer, seed=seed, n_steps=1, threads=threads)
+    if workload == "cfg2":
+        return hi.cfg2(layer, seed=seed, threads=threads)
+    if workload == "cfg3":
+        return hi.cfg3(layer, seed=seed, threads=threads)
+    if workload == "cfg4":
+        return hi.cfg4(0.10, 0.5, 32, seed=seed, layer=layer, threads=threads)
+    raise SystemExit(f"unknown workload {workload}")
+
+
+WORKLOAD_TEXT = {
+    "cfg0": "1 layer, B=1, 2048 tokens, 2 static / 2 dynamic heads, budget 10%, chunk 32",
+    "cfg1": "28 layers, B=1, 16384 tokens (image blocks), static fraction 0.5, budget 10%, chunk 32",
+    "cfg2": "28 layers, B=4, 24K-32K tokens (64 frames x 500 video-like), static fraction 0.6, budget 10%, chunk 64",
+    "cfg3": "28 layers, B=8, 50000 tokens, static fraction 0.4, budget 5%, chunk 32, planted chunks",
+    "cfg4": "1 layer, B=16, 32768 tokens, cell budget 10% / static fraction 0.5 / chunk 32",
+}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_decode_timing(L, budget_s: float):
+    """Times the oracle's decode step (score + select + attend, all heads of one layer) as it stands."""
+    from oracle import hkv_oracle as o
+    dyn = [(b, h) for b in range(L.batch) for h in range(L.n_kv_heads)]
+    # compression is set-up for the decode timing; window scores are skipped through a score override
+    ts = np.zeros((L.batch, L.n_kv_heads, L.max_seq_len), dtype=np.float32)
+    ts[:] = np.linspace(1.0, 0.0, L.max_seq_len, dtype=np.float32)[None, None, :]
+    oc = o.compress_layer(L, token_scores=ts, only=dyn)
+    t0, n = time.perf_counter(), 0
+    while True:
+        o.decode_layer(L, oc, L.q[0])
+        n += 1
+        if time.perf_counter() - t0 > budget_s or n >= 50:
+            break
+    return (time.perf_counter() - t0) / n, n
+
+
+def layer_algo_bytes(L) -> int:
+    """512 B per retained token + 256 B per chunk mean (host arithmetic on the plan inputs)."""
+    tot = 0
+    cs = L.chunk_size
+    for b in range(L.batch):
+        C = int(L.seq_lens[b])
+        for h in range(L.n_kv_heads):
+            bud = min(int(L.budgets[b, h]), C)
+            if L.head_type[b, h] == 0:
+                tot += 512 * bud
+            else:
+                nch = (C + cs - 1) // cs
+                k = min(nch, (bud + cs - 1) // cs)
+                tot += 512 * min(k * cs, C) + 256 * nch
+    return tot
+
+
+def run_reference(args):
+    """The reference arm of this tier is the CPU oracle, timed as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = min(os.cpu_count() or 8, 32)
+    L = layer_inputs(args.workload, 0, args.seed, threads)
+    n_layers = N_LAYERS[args.workload]
+    per = []
+    for i in range(args.warmup + args.steps):
+        dt, _ = oracle_decode_timing(L, 0.0)          # one decode of one layer per step (bounded sample)
+        if i >= args.warmup:
+            per.append(dt)
+    t = sum(per) / len(per)
+    bytes_layer = layer_algo_bytes(L)
+    value = bytes_layer / t / 1e9
+    sample = f"1 of {n_layers} layers per step (all {L.batch * L.n_kv_heads} heads), oracle decode_layer, step time scaled x{n_layers}"
+    line = {"impl": "reference", "metric": "decode_attention_achieved_hbm_GBps", "value": value, "unit": "GB/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * n_layers * 1e3,
+            "us_per_step": t * n_layers * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}"},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=list(N_LAYERS))
+    ap.add_argument("--seed", type=int, default=2)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time spent on the oracle baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2604_05887_b200 import binding as hkv          # raises if libhkv.so is missing: no fallback
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA path has no CPU fallback)")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    # ---- build the workload: generate each layer on the host, upload, compress, keep the cache ----
+    n_layers = N_LAYERS[args.workload]
+    threads = min(os.cpu_count() or 8, 32)
+    caches, qs, outs, L0 = [], [], [], None
+    t_gen = t_comp = 0.0
+    kv_in_bytes = 0
+    for layer in range(n_layers):
+        t0 = time.perf_counter()
+        L = layer_inputs(args.workload, layer, args.seed + 1000 * rank, threads)
+        t_gen += time.perf_counter() - t0
+        k_dev, v_dev = to_device_bf16(L.k, dev), to_device_bf16(L.v, dev)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        lc = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
+        e1.record()
+        torch.cuda.synchronize()
+        t_comp += e0.elapsed_time(e1) * 1e-3
+        kv_in_bytes += sum(int(c) for c in L.seq_lens) * L.n_kv_heads * 512
+        caches.append(lc)
+        qs.append(to_device_bf16(L.q[0], dev))
+        outs.append(lc.new_out())
+        if layer == 0:
+            L0 = L
+        else:
+            del L
+        del k_dev, v_dev
+    stats = [c.stats for c in caches]
+    algo_bytes = sum(s["algorithmic_bytes_per_step"] for s in stats)
+    attend_bytes = sum(512 * s["retained_tokens"] for s in stats)
+    launches_per_step = sum(s["launches_per_decode"] for s in stats)
+    resident = sum(s["cache_bytes"] for s in stats)
+
+    def step():
+        for lc, q, o_ in zip(caches, qs, outs):
+            hkv.hkv_decode_attn(lc.handle, q, o_)
+
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            step()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step()
+
+        # end-to-end variant: the step's queries start in pinned host memory, outputs end there
+        q_host = torch.stack([q.cpu() for q in qs]).pin_memory()
+        out_host = torch.empty((n_layers,) + tuple(outs[0].shape), dtype=outs[0].dtype).pin_memory()
+        q_all = torch.empty_like(q_host, device=dev)
+        out_all = torch.empty_like(out_host, device=dev)
+
+        def step_e2e():
+            q_all.copy_(q_host, non_blocking=True)
+            for i, lc in enumerate(caches):
+                hkv.hkv_decode_attn(lc.handle, q_all[i], out_all[i])
+            out_host.copy_(out_all, non_blocking=True)
+
+        step_e2e()
+        stream.synchronize()
+        graph_e2e = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_e2e, stream=stream):
+            step_e2e()
+        stream.synchronize()
+
+        def barrier():
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        def timed(g, n):
+            barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(n):
+                g.replay()
+            b.record(stream)
+            barrier()
+            ms = a.elapsed_time(b)
+            if dist is not None:
+                t = torch.tensor([ms], device=dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            return ms
+
+        for _ in range(max(args.warmup, 3)):
+            graph.replay()
+        with ClockSampler(local) as clk:
+            ms = timed(graph, args.steps)
+        for _ in range(3):
+            graph_e2e.replay()
+        ms_e2e = timed(graph_e2e, args.steps)
+
+        # ---- per-launch duration of the dominant kernel (flash-decode), CUDA events on its stream ----
+        for lc, q in zip(caches, qs):
+            hkv.hkv_select_chunks(lc.handle, q)
+        reps = max(3, min(20, args.steps))
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(reps * n_layers)]
+        sel_evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(reps * n_layers)]
+        i = 0
+        for _ in range(reps):
+            for lc, q, o_ in zip(caches, qs, outs):
+                sel_evs[i][0].record(stream)
+                hkv.hkv_select_chunks(lc.handle, q)
+                sel_evs[i][1].record(stream)
+                evs[i][0].record(stream)
+                hkv.hkv_attend(lc.handle, q, o_)
+                evs[i][1].record(stream)
+                i += 1
+        stream.synchronize()
+        attend_ms = [a.elapsed_time(b) for a, b in evs[n_layers:]]        # first pass is warm-up
+        select_ms = [a.elapsed_time(b) for a, b in sel_evs[n_layers:]]
+        code, detail = hkv.hkv_last_device_error(caches[0].handle)
+
+    world_bytes = algo_bytes * world          # every rank runs a replica of the same size (weak scaling)
+    t_step = ms * 1e-3 / args.steps
+    value = world_bytes / t_step / 1e9
+    peak, peak_src = measured_peak()
+    attend_avg_s = (sum(attend_ms) / len(attend_ms)) * 1e-3
+    achieved = (attend_bytes / n_layers) / attend_avg_s / 1e9
+    t_e2e = ms_e2e * 1e-3 / args.steps
+    h2d = q_host.numel() * q_host.element_size()
+    d2h = out_host.numel() * out_host.element_size()
+
+    line = {
+        "metric": "decode_attention_achieved_hbm_GBps", "value": value, "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": t_step * 1e3,
+        "us_per_step": t_step * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}", "layers": n_layers,
+                   "algorithmic_bytes_per_step": algo_bytes, "resident_cache_bytes": resident,
+                   "l2": "inputs larger than L2: one step streams %.0f MB of distinct KV" % (algo_bytes / 1e6)
+                   if algo_bytes > 2 * 126e6 else "WARNING: step working set near L2 size",
+                   "launch": "CUDA graph of one hkv_decode_attn per layer, layers in sequence",
+                   "compress_GBps_of_input_kv": kv_in_bytes / t_comp / 1e9},
+        "frac_of_measured_peak": value / world / peak, "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "hbm", "kernel": "flash_decode_kernel (per layer launch)", "achieved": achieved,
+                     "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                     "avg_launch_us": attend_avg_s * 1e6, "bytes_per_launch": attend_bytes / n_layers,
+                     "select_kernel_avg_launch_us": 1e3 * sum(select_ms) / len(select_ms),
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
+        "e2e": {"value": world_bytes / t_e2e / 1e9, "unit": "GB/s", "us_per_step": t_e2e * 1e6,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "how": "pinned host queries -> device, 28 x hkv_decode_attn, outputs -> pinned host, all inside the timed graph"},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clk.summary(),
+        "device_error": [code, detail],
+        "paper_context": "paper reports 7.9x KV-memory reduction and 1.52x decode speed-up (whole model, NVIDIA L40S); no attention-only number",
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        dt, n = oracle_decode_timing(L0, args.cpu_seconds)
+        b0 = stats[0]["algorithmic_bytes_per_step"]
+        line["cpu_baseline"] = {"value": b0 / dt / 1e9, "unit": "GB/s", "us_per_step": dt * n_layers * 1e6,
+                                "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"oracle decode_layer on layer 0 of {n_layers} ({L0.batch * L0.n_kv_heads} heads), "
+                                          f"{n} repetitions, step time scaled x{n_layers}"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

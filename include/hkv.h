@@ -139,6 +139,23 @@ hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* str
 hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q, void* const* out,
                                  int32_t n, void* stream);
 
+/* The two stages of hkv_decode_attn as separate calls (hkv_decode_attn = hkv_select_chunks followed
+ * by hkv_attend on the same stream).  hkv_select_chunks scores every chunk of every dynamic head
+ * against q and stores the top-k chunk ids in the cache (Appendix A: "identify relevant chunks by
+ * computing the inner product between the query vector and chunk metadata").  hkv_attend runs the
+ * attention of all heads over the static cache and the currently stored selection (Appendix A: "The
+ * final attention output is then computed together with the static KV cache"); it needs one earlier
+ * hkv_select_chunks (or hkv_decode_attn) if the cache has dynamic heads.  Same pointer rules. */
+hkv_status hkv_select_chunks(hkv_cache* cache, const void* q, void* stream);
+hkv_status hkv_attend(hkv_cache* cache, const void* q, void* out, void* stream);
+
+/* hkv_decode_attn with HOST buffers: copies q_host -> q_dev, runs the step, copies out_dev ->
+ * out_host, all enqueued on `stream` (the result is in out_host once the stream has passed the call).
+ *   q_host, out_host  host memory (pinned for truly asynchronous copies), shapes as q / out
+ *   q_dev, out_dev    caller-owned device staging buffers of the same sizes */
+hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_host, void* q_dev,
+                                void* out_dev, void* stream);
+
 hkv_status hkv_cache_destroy(hkv_cache* cache);
 
 /* ---- introspection (parity tests, roofline numerator). These synchronise the given stream. ---- */

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "HKV_OK", 1: "HKV_ERR_INVALID_ARG", 2: "HKV_ERR_SHAPE", 3: "H
                 4: "HKV_ERR_WORKSPACE", 5: "HKV_ERR_UNSUPPORTED", 6: "HKV_ERR_CUDA", 7: "HKV_ERR_TIMEOUT",
                 8: "HKV_ERR_INDEX"}
 
-EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi", "hkv_cache_destroy",
+EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi", "hkv_select_chunks",
+           "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string"]
 
@@ -62,6 +63,9 @@ def _load() -> C.CDLL:
                                  C.POINTER(vp)]
     lib.hkv_decode_attn.argtypes = [vp, vp, vp, vp]
     lib.hkv_decode_attn_multi.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int32, vp]
+    lib.hkv_select_chunks.argtypes = [vp, vp, vp]
+    lib.hkv_attend.argtypes = [vp, vp, vp, vp]
+    lib.hkv_decode_attn_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hkv_cache_destroy.argtypes = [vp]
     for name in ("hkv_get_static_indices", "hkv_get_selected_chunks"):
         getattr(lib, name).argtypes = [vp, C.c_int32, C.c_int32, i32p, C.c_int32, i32p, vp]
@@ -158,6 +162,22 @@ def hkv_decode_attn_multi(caches: Sequence[int], qs, outs, stream=None) -> None:
     arr = C.c_void_p * n
     _check(lib.hkv_decode_attn_multi(arr(*caches), arr(*[_dev(t) for t in qs]), arr(*[_dev(t) for t in outs]),
                                      n, _stream(stream)), "hkv_decode_attn_multi")
+
+
+def hkv_select_chunks(cache: int, q, stream=None) -> None:
+    _check(lib.hkv_select_chunks(cache, _dev(q), _stream(stream)), "hkv_select_chunks")
+
+
+def hkv_attend(cache: int, q, out, stream=None) -> None:
+    _check(lib.hkv_attend(cache, _dev(q), _dev(out), _stream(stream)), "hkv_attend")
+
+
+def hkv_decode_attn_host(cache: int, q_host, out_host, q_dev, out_dev, stream=None) -> None:
+    """q_host / out_host: CPU torch tensors (pinned for asynchronous copies); q_dev / out_dev: CUDA staging."""
+    if q_host.is_cuda or out_host.is_cuda or not q_host.is_contiguous() or not out_host.is_contiguous():
+        raise ValueError("q_host and out_host must be contiguous CPU tensors")
+    _check(lib.hkv_decode_attn_host(cache, q_host.data_ptr(), out_host.data_ptr(), _dev(q_dev), _dev(out_dev),
+                                    _stream(stream)), "hkv_decode_attn_host")
 
 
 def hkv_cache_destroy(cache: int) -> None:

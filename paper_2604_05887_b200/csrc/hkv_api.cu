@@ -254,30 +254,38 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
   }
 }
 
-hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
-                                 void* stream) {
-  if (!caches || !q || !out || n < 1 || n > kMaxMulti) return HKV_ERR_INVALID_ARG;
+static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
+                                void* stream, bool do_select, bool do_attend) {
+  if (!caches || !q || n < 1 || n > kMaxMulti || (do_attend && !out)) return HKV_ERR_INVALID_ARG;
   DecodeBatch batch;
   std::memset(&batch, 0, sizeof(batch));
   batch.n = n;
   for (int i = 0; i < n; ++i) {
     const hkv_cache* c = caches[i];
-    if (!c || !q[i] || !out[i]) return HKV_ERR_INVALID_ARG;
+    if (!c || !q[i] || (do_attend && !out[i])) return HKV_ERR_INVALID_ARG;
     if (c->hdr.group != caches[0]->hdr.group || ((c->hdr.flags ^ caches[0]->hdr.flags) & HKV_OUT_F32)) return HKV_ERR_SHAPE;
     batch.cache[i] = c->dev_base;
     batch.q[i] = q[i];
-    batch.out[i] = out[i];
+    batch.out[i] = do_attend ? out[i] : nullptr;
     batch.split_prefix[i + 1] = batch.split_prefix[i] + c->hdr.n_splits;
     batch.dyn_prefix[i + 1] = batch.dyn_prefix[i] + c->hdr.n_dynamic;
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (launch_select_chunks(batch, batch.dyn_prefix[n], s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
-  if (launch_flash_decode(batch, batch.split_prefix[n], caches[0]->hdr.group, (caches[0]->hdr.flags & HKV_OUT_F32) != 0, s) !=
-      cudaSuccess) {
+  if (do_select && launch_select_chunks(batch, batch.dyn_prefix[n], s) != cudaSuccess) {
+    cudaGetLastError();
+    return HKV_ERR_CUDA;
+  }
+  if (do_attend && launch_flash_decode(batch, batch.split_prefix[n], caches[0]->hdr.group,
+                                       (caches[0]->hdr.flags & HKV_OUT_F32) != 0, s) != cudaSuccess) {
     cudaGetLastError();
     return HKV_ERR_CUDA;
   }
   return HKV_OK;
+}
+
+hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
+                                 void* stream) {
+  return decode_stages(caches, q, out, n, stream, true, true);
 }
 
 hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* stream) {
@@ -285,7 +293,35 @@ hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* str
   hkv_cache* one[1] = {cache};
   const void* qs[1] = {q};
   void* os[1] = {out};
-  return hkv_decode_attn_multi(one, qs, os, 1, stream);
+  return decode_stages(one, qs, os, 1, stream, true, true);
+}
+
+hkv_status hkv_select_chunks(hkv_cache* cache, const void* q, void* stream) {
+  if (!cache) return HKV_ERR_INVALID_ARG;
+  hkv_cache* one[1] = {cache};
+  const void* qs[1] = {q};
+  return decode_stages(one, qs, nullptr, 1, stream, true, false);
+}
+
+hkv_status hkv_attend(hkv_cache* cache, const void* q, void* out, void* stream) {
+  if (!cache) return HKV_ERR_INVALID_ARG;
+  hkv_cache* one[1] = {cache};
+  const void* qs[1] = {q};
+  void* os[1] = {out};
+  return decode_stages(one, qs, os, 1, stream, false, true);
+}
+
+hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_host, void* q_dev, void* out_dev,
+                                void* stream) {
+  if (!cache || !q_host || !out_host || !q_dev || !out_dev) return HKV_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t n = static_cast<size_t>(cache->cfg.batch) * cache->cfg.n_q_heads * cache->cfg.head_dim;
+  const size_t out_elt = (cache->hdr.flags & HKV_OUT_F32) ? 4 : 2;
+  if (cudaMemcpyAsync(q_dev, q_host, n * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  hkv_status st = hkv_decode_attn(cache, q_dev, out_dev, stream);
+  if (st != HKV_OK) return st;
+  if (cudaMemcpyAsync(out_host, out_dev, n * out_elt, cudaMemcpyDeviceToHost, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  return HKV_OK;
 }
 
 hkv_status hkv_cache_destroy(hkv_cache* cache) {
