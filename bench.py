@@ -203,6 +203,9 @@ def main():
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time spent on the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="use only the first N layers of the workload (small case for profiler captures; "
+                         "the line is then marked reduced and is not the headline number)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -226,6 +229,8 @@ def main():
 
     # ---- build the workload: generate each layer on the host, upload, compress, keep the cache ----
     n_layers = N_LAYERS[args.workload]
+    if args.layers > 0:
+        n_layers = min(n_layers, args.layers)
     threads = min(os.cpu_count() or 8, 32)
     caches, qs, outs, L0 = [], [], [], None
     t_gen = t_comp = 0.0
@@ -253,7 +258,6 @@ def main():
         del k_dev, v_dev
     stats = [c.stats for c in caches]
     algo_bytes = sum(s["algorithmic_bytes_per_step"] for s in stats)
-    attend_bytes = sum(512 * s["retained_tokens"] for s in stats)
     launches_per_step = sum(s["launches_per_decode"] for s in stats)
     resident = sum(s["cache_bytes"] for s in stats)
 
@@ -318,35 +322,36 @@ def main():
             graph_e2e.replay()
         ms_e2e = timed(graph_e2e, args.steps)
 
-        # ---- per-launch duration of the dominant kernel (flash-decode), CUDA events on its stream ----
-        for lc, q in zip(caches, qs):
-            hkv.hkv_select_chunks(lc.handle, q)
+        # ---- per-launch duration of the dominant kernel (the fused decode kernel, one launch per
+        # layer), CUDA events on its stream around every launch; the selection-only and attention-only
+        # phases of the same kernel are timed the same way for the breakdown ----
         reps = max(3, min(20, args.steps))
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-               for _ in range(reps * n_layers)]
-        sel_evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+
+        def per_launch(fn):
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                    for _ in range(reps * n_layers)]
-        i = 0
-        for _ in range(reps):
-            for lc, q, o_ in zip(caches, qs, outs):
-                sel_evs[i][0].record(stream)
-                hkv.hkv_select_chunks(lc.handle, q)
-                sel_evs[i][1].record(stream)
-                evs[i][0].record(stream)
-                hkv.hkv_attend(lc.handle, q, o_)
-                evs[i][1].record(stream)
-                i += 1
-        stream.synchronize()
-        attend_ms = [a.elapsed_time(b) for a, b in evs[n_layers:]]        # first pass is warm-up
-        select_ms = [a.elapsed_time(b) for a, b in sel_evs[n_layers:]]
+            i = 0
+            for _ in range(reps):
+                for lc, q, o_ in zip(caches, qs, outs):
+                    evs[i][0].record(stream)
+                    fn(lc, q, o_)
+                    evs[i][1].record(stream)
+                    i += 1
+            stream.synchronize()
+            ms_ = [a.elapsed_time(b) for a, b in evs[n_layers:]]        # first pass is warm-up
+            return sum(ms_) / len(ms_)
+
+        fused_ms = per_launch(lambda lc, q, o_: hkv.hkv_decode_attn(lc.handle, q, o_))
+        select_ms = per_launch(lambda lc, q, o_: hkv.hkv_select_chunks(lc.handle, q))
+        attend_ms = per_launch(lambda lc, q, o_: hkv.hkv_attend(lc.handle, q, o_))
         code, detail = hkv.hkv_last_device_error(caches[0].handle)
 
     world_bytes = algo_bytes * world          # every rank runs a replica of the same size (weak scaling)
     t_step = ms * 1e-3 / args.steps
     value = world_bytes / t_step / 1e9
     peak, peak_src = measured_peak()
-    attend_avg_s = (sum(attend_ms) / len(attend_ms)) * 1e-3
-    achieved = (attend_bytes / n_layers) / attend_avg_s / 1e9
+    fused_avg_s = fused_ms * 1e-3
+    achieved = (algo_bytes / n_layers) / fused_avg_s / 1e9
     t_e2e = ms_e2e * 1e-3 / args.steps
     h2d = q_host.numel() * q_host.element_size()
     d2h = out_host.numel() * out_host.element_size()
@@ -356,17 +361,21 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": t_step * 1e3,
         "us_per_step": t_step * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}", "layers": n_layers,
+        "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}"
+                   + (f" -- REDUCED to {n_layers} layers (profiling case)" if n_layers != N_LAYERS[args.workload] else ""),
+                   "layers": n_layers,
                    "algorithmic_bytes_per_step": algo_bytes, "resident_cache_bytes": resident,
                    "l2": "inputs larger than L2: one step streams %.0f MB of distinct KV" % (algo_bytes / 1e6)
                    if algo_bytes > 2 * 126e6 else "WARNING: step working set near L2 size",
                    "launch": "CUDA graph of one hkv_decode_attn per layer, layers in sequence",
                    "compress_GBps_of_input_kv": kv_in_bytes / t_comp / 1e9},
         "frac_of_measured_peak": value / world / peak, "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
-        "roofline": {"bound": "hbm", "kernel": "flash_decode_kernel (per layer launch)", "achieved": achieved,
-                     "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                     "avg_launch_us": attend_avg_s * 1e6, "bytes_per_launch": attend_bytes / n_layers,
-                     "select_kernel_avg_launch_us": 1e3 * sum(select_ms) / len(select_ms),
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel (score + top-k + flash-decode + merge, one launch per layer)",
+                     "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
+                     "avg_launch_us": fused_avg_s * 1e6, "bytes_per_launch": algo_bytes / n_layers,
+                     "in_graph_us_per_launch": t_step * 1e6 / n_layers,
+                     "select_only_avg_launch_us": select_ms * 1e3, "attend_only_avg_launch_us": attend_ms * 1e3,
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
         "e2e": {"value": world_bytes / t_e2e / 1e9, "unit": "GB/s", "us_per_step": t_e2e * 1e6,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -56,7 +56,6 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
   }
   c.cfg = *cfg;
   c.units.clear();
-  c.splits.clear();
   Header& H = c.hdr;
   std::memset(&H, 0, sizeof(H));
   H.batch = B; H.n_q_heads = cfg->n_q_heads; H.n_kv_heads = Hkv; H.group = G;
@@ -101,46 +100,16 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
     }
   }
 
-  // ---- splits: one wave of CTAs whenever the work allows it ----
-  const int target = sm_count();
-  int max_tiles = 1;
-  for (auto& u : c.units) max_tiles = std::max(max_tiles, (u.n_tok + kTile - 1) / kTile);
-  int tps = kDecWarps;
-  while (tps < max_tiles) {
-    int64_t n = 0;
-    for (auto& u : c.units) n += ((u.n_tok + kTile - 1) / kTile + tps - 1) / tps;
-    if (n <= target) break;
-    tps += kDecWarps;
-  }
-  int split_total = 0;
-  for (int pass = 0; pass < 2; ++pass) {     // static units first: their work does not wait for the selection
-    for (int i = 0; i < H.n_units; ++i) {
-      Unit& u = c.units[i];
-      if (u.type != pass) continue;
-      const int tiles = (u.n_tok + kTile - 1) / kTile;
-      u.n_splits = std::max(1, (tiles + tps - 1) / tps);
-      u.split_base = split_total;
-      for (int s = 0; s < u.n_splits; ++s) {
-        Split sp;
-        sp.unit = i; sp.tile_begin = s * tps; sp.tile_end = std::min(tiles, (s + 1) * tps); sp.slot = s;
-        c.splits.push_back(sp);
-      }
-      split_total += u.n_splits;
-    }
-  }
-  H.n_splits = split_total;
+  c.max_tiles = 1;
+  for (auto& u : c.units) c.max_tiles = std::max(c.max_tiles, (u.n_tok + kTile - 1) / kTile);
 
   // ---- cache_mem layout ----
-  int64_t off = align_up(sizeof(Header));
-  H.units_off = off;     off = align_up(off + sizeof(Unit) * H.n_units);
-  H.splits_off = off;    off = align_up(off + sizeof(Split) * split_total);
+  int64_t off = kUnitsOff;
+  off = align_up(off + sizeof(Unit) * H.n_units);
   H.dyn_list_off = off;  off = align_up(off + 4ll * std::max(1, H.n_dynamic));
   H.sta_list_off = off;  off = align_up(off + 4ll * std::max(1, H.n_static));
-  const int64_t tables_end = off;
-  H.counters_off = off;  off = align_up(off + 4ll * H.n_units);
-  H.n_valid_off = off;   off = align_up(off + 4ll * H.n_units);
+  H.n_valid_off = off;   off = align_up(off + 4ll * H.n_units);   // tables end here; the rest starts at zero
   H.err_off = off;       off = align_up(off + 8);
-  H.partials_off = off;  off = align_up(off + 4ll * split_total * G * (kHeadDim + 2));
   for (auto& u : c.units) {
     u.idx_off = off;
     off = align_up(off + 4ll * std::max(1, u.type == 0 ? u.n_tok : u.k_sel));
@@ -154,7 +123,6 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
     u.v_off = off;  off = align_up(off + static_cast<int64_t>(kRowBytes) * u.plane_rows);
   }
   c.cache_bytes = static_cast<size_t>(off);
-  (void)tables_end;
 
   // ---- workspace layout: s_w per static unit, then the row statistics of the window softmax ----
   int64_t woff = 0;
@@ -222,19 +190,18 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
     const Header& H = c->hdr;
 
     // tables: one host image, one copy
-    const size_t tables = static_cast<size_t>(H.counters_off);
+    const size_t tables = static_cast<size_t>(H.n_valid_off);
     std::vector<char> img(tables, 0);
     std::memcpy(img.data(), &H, sizeof(H));
-    std::memcpy(img.data() + H.units_off, c->units.data(), sizeof(Unit) * c->units.size());
-    std::memcpy(img.data() + H.splits_off, c->splits.data(), sizeof(Split) * c->splits.size());
+    std::memcpy(img.data() + kUnitsOff, c->units.data(), sizeof(Unit) * c->units.size());
     int32_t* dl = reinterpret_cast<int32_t*>(img.data() + H.dyn_list_off);
     int32_t* sl = reinterpret_cast<int32_t*>(img.data() + H.sta_list_off);
     for (int i = 0; i < H.n_units; ++i) {
       if (c->units[i].type) *dl++ = i; else *sl++ = i;
     }
     bool ok = cudaMemcpyAsync(c->dev_base, img.data(), tables, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    // counters, n_valid, error word start at zero
-    ok = ok && cudaMemsetAsync(c->dev_base + H.counters_off, 0, static_cast<size_t>(H.partials_off - H.counters_off), s) ==
+    // n_valid and the error word start at zero
+    ok = ok && cudaMemsetAsync(c->dev_base + H.n_valid_off, 0, static_cast<size_t>(H.err_off + 8 - H.n_valid_off), s) ==
                    cudaSuccess;
     if (ok && H.n_static > 0) {
       if (!token_scores)
@@ -257,26 +224,38 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
 static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
                                 void* stream, bool do_select, bool do_attend) {
   if (!caches || !q || n < 1 || n > kMaxMulti || (do_attend && !out)) return HKV_ERR_INVALID_ARG;
-  DecodeBatch batch;
-  std::memset(&batch, 0, sizeof(batch));
-  batch.n = n;
+  DecodeParams P;
+  std::memset(&P, 0, sizeof(P));
+  P.n = n;
+  int max_tiles = 1, n_dynamic = 0;
   for (int i = 0; i < n; ++i) {
     const hkv_cache* c = caches[i];
     if (!c || !q[i] || (do_attend && !out[i])) return HKV_ERR_INVALID_ARG;
-    if (c->hdr.group != caches[0]->hdr.group || ((c->hdr.flags ^ caches[0]->hdr.flags) & HKV_OUT_F32)) return HKV_ERR_SHAPE;
-    batch.cache[i] = c->dev_base;
-    batch.q[i] = q[i];
-    batch.out[i] = do_attend ? out[i] : nullptr;
-    batch.split_prefix[i + 1] = batch.split_prefix[i] + c->hdr.n_splits;
-    batch.dyn_prefix[i + 1] = batch.dyn_prefix[i] + c->hdr.n_dynamic;
+    const Header& H = c->hdr;
+    const Header& H0 = caches[0]->hdr;
+    if (H.group != H0.group || H.n_q_heads != H0.n_q_heads || H.n_kv_heads != H0.n_kv_heads ||
+        H.chunk_size != H0.chunk_size || H.scale != H0.scale || ((H.flags ^ H0.flags) & HKV_OUT_F32))
+      return HKV_ERR_SHAPE;
+    P.cache[i] = c->dev_base;
+    P.q[i] = q[i];
+    P.out[i] = do_attend ? out[i] : nullptr;
+    P.n_valid_off[i] = H.n_valid_off;
+    P.err_off[i] = H.err_off;
+    P.unit_prefix[i + 1] = P.unit_prefix[i] + H.n_units;
+    max_tiles = std::max(max_tiles, c->max_tiles);
+    n_dynamic += H.n_dynamic;
   }
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (do_select && launch_select_chunks(batch, batch.dyn_prefix[n], s) != cudaSuccess) {
-    cudaGetLastError();
-    return HKV_ERR_CUDA;
-  }
-  if (do_attend && launch_flash_decode(batch, batch.split_prefix[n], caches[0]->hdr.group,
-                                       (caches[0]->hdr.flags & HKV_OUT_F32) != 0, s) != cudaSuccess) {
+  if (!do_attend && n_dynamic == 0) return HKV_OK;   // nothing to select
+  const Header& H0 = caches[0]->hdr;
+  P.group = H0.group; P.n_q_heads = H0.n_q_heads; P.n_kv_heads = H0.n_kv_heads; P.chunk_size = H0.chunk_size;
+  P.scale_log2e = H0.scale * 1.4426950408889634f;
+  P.phase = (do_select ? kPhaseSelect : 0u) | (do_attend ? kPhaseAttend : 0u);
+  P.out_f32 = (H0.flags & HKV_OUT_F32) ? 1u : 0u;
+  int max_cluster = 1;
+  if (decode_max_cluster(P.group, &max_cluster) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  const int total_units = P.unit_prefix[n];
+  P.cluster = std::min(max_cluster, choose_cluster(total_units, max_tiles, sm_count()));
+  if (launch_decode(P, total_units, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
     cudaGetLastError();
     return HKV_ERR_CUDA;
   }
@@ -366,8 +345,17 @@ hkv_status hkv_get_summaries(hkv_cache* c, int32_t b, int32_t h, uint16_t* host_
   if (u.type != 1) return HKV_ERR_INVALID_ARG;
   *n_chunks = u.n_chunks;
   if (capacity_rows < u.n_chunks) return HKV_ERR_WORKSPACE;
-  return d2h(host_out, c->dev_base + u.summ_off, static_cast<size_t>(kRowBytes) * u.n_chunks,
-             static_cast<cudaStream_t>(stream));
+  hkv_status st = d2h(host_out, c->dev_base + u.summ_off, static_cast<size_t>(kRowBytes) * u.n_chunks,
+                      static_cast<cudaStream_t>(stream));
+  if (st != HKV_OK) return st;
+  // rows are held with their 16-byte pieces permuted by (row & 7): put them back in order
+  for (int r = 0; r < u.n_chunks; ++r) {
+    uint16_t* row = host_out + static_cast<size_t>(r) * kHeadDim;
+    uint16_t tmp[kHeadDim];
+    std::memcpy(tmp, row, sizeof(tmp));
+    for (int p = 0; p < 16; ++p) std::memcpy(row + p * 8, tmp + ((p ^ (r & 7)) * 8), 16);
+  }
+  return HKV_OK;
 }
 
 hkv_status hkv_window_scores_offset(const hkv_cache* c, int32_t b, int32_t h, size_t* offset) {
@@ -389,8 +377,8 @@ hkv_status hkv_cache_stats(const hkv_cache* c, hkv_stats* st) {
   st->workspace_bytes = static_cast<int64_t>(c->workspace_bytes);
   st->n_static = c->hdr.n_static;
   st->n_dynamic = c->hdr.n_dynamic;
-  st->n_splits = c->hdr.n_splits;
-  st->launches_per_decode = 1 + (c->hdr.n_dynamic > 0 ? 1 : 0);
+  st->n_splits = c->hdr.n_units * choose_cluster(c->hdr.n_units, c->max_tiles, sm_count());
+  st->launches_per_decode = 1;
   return HKV_OK;
 }
 

@@ -19,7 +19,7 @@ __device__ __forceinline__ const Unit* unit_of(const char* cache, const Header* 
   const int32_t* list = reinterpret_cast<const int32_t*>(cache + (dynamic ? hdr->dyn_list_off : hdr->sta_list_off));
   const int uid = list[ordinal];
   if (uid_out) *uid_out = uid;
-  return reinterpret_cast<const Unit*>(cache + hdr->units_off) + uid;
+  return reinterpret_cast<const Unit*>(cache + kUnitsOff) + uid;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -231,7 +231,8 @@ __global__ void __launch_bounds__(kKeepThreads)
   if (budget <= w) {
     const int start = C - budget;
     emitted = block_select_emit(
-        C, 0, [](int) { return 0u; }, [&](int i) { return i >= start; }, out, hist, wsum, bc);
+        C, 0, [](int) { return 0u; }, [&](int i) { return i >= start; }, [&](int pos, int i) { out[pos] = i; }, hist, wsum,
+        bc);
   } else {
     const int room = budget - w;
     const bool rank_text = n_text >= room;       // window + text do not fit: rank the text tokens
@@ -243,7 +244,8 @@ __global__ void __launch_bounds__(kKeepThreads)
           const bool is_t = txt[i] != 0;
           return (is_t == rank_text) ? float_key(scores[i]) : 0u;
         },
-        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, out, hist, wsum, bc);
+        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, [&](int pos, int i) { out[pos] = i; }, hist,
+        wsum, bc);
   }
   if (tid == 0) {
     reinterpret_cast<int32_t*>(cache + hdr->n_valid_off)[uid] = emitted;
@@ -299,7 +301,9 @@ __global__ void __launch_bounds__(kHeadDim) chunk_means_kernel(char* cache, cons
     const int t0 = c * cs, t1 = min(t0 + cs, C);
     float acc = 0.f;
     for (int tk = t0; tk < t1; ++tk) acc = __fadd_rn(acc, __bfloat162float(kp[static_cast<size_t>(tk) * kHeadDim + d]));
-    out[static_cast<size_t>(c) * kHeadDim + d] = __float2bfloat16_rn(__fdiv_rn(acc, static_cast<float>(t1 - t0)));
+    // 16-byte piece p of chunk c is stored at position p ^ (c & 7), like K/V rows
+    out[static_cast<size_t>(c) * kHeadDim + ((((d >> 3) ^ (c & 7)) << 3) | (d & 7))] =
+        __float2bfloat16_rn(__fdiv_rn(acc, static_cast<float>(t1 - t0)));
   }
 }
 

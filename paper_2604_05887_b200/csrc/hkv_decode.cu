@@ -1,5 +1,33 @@
-// Decode-step kernels: chunk scoring + exact top-k chunk selection for dynamic heads, and the
-// split-K flash-decode over each head's retained token list with the split merge fused in.
+// The decode-step kernel: for every (sequence, kv head) unit, chunk scoring and exact top-k chunk
+// selection (dynamic heads), flash-decoding over the unit's retained token list, and the merge of
+// the partial results — one launch per layer.
+//
+// Work decomposition.  A thread-block CLUSTER of `cluster` CTAs owns one unit.  Inside a CTA every
+// warp is an independent consumer with its own ring of kDecStages staging buffers and its own
+// mbarriers; the TMA engine fills the ring with 1-D bulk copies (no multicast).
+//
+//   dynamic unit, selection:  the cluster's CTAs split the unit's chunk means between them; a warp
+//     stages 64 means at a time and computes  S^T = M Q^T  (rows = chunks, columns = the group's
+//     query heads) on tensor cores; the chunk score is the float32 sum over the group's heads.
+//     Scores are pushed into the shared memory of every CTA of the cluster (distributed shared
+//     memory), a cluster barrier follows, and each CTA then runs the same exact radix selection on
+//     its own copy, so that every CTA knows the ascending list of selected chunks without a
+//     round trip through global memory.
+//   every unit, attention:  the unit's token list (static: the compacted rows; dynamic: the rows of
+//     the selected chunks) is cut into 32-token tiles, dealt to the cluster's CTAs as contiguous
+//     ranges and to a CTA's warps round-robin.  Per tile:  S^T = K Q^T  (rows = tokens, columns =
+//     query heads, so the group shares every loaded KV tile and no tensor-core row is padding),
+//     online softmax in float32 (base-2 exponent), P^T moved into operand layout with movmatrix,
+//     O^T += V^T P^T.
+//   merge:  the warps of a CTA are combined in shared memory; the CTAs of the cluster read each
+//     other's partial (m, l, O) through distributed shared memory, CTA r producing output rows
+//     r, r + cluster, ... — fixed order, no atomics, deterministic.
+//
+// K/V rows and chunk means live in HBM with their sixteen 16-byte pieces XOR-permuted by (row & 7),
+// which makes the ldmatrix reads of a staged tile bank-conflict free without any copy in shared
+// memory.
+#include <cstring>
+
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
 
@@ -7,142 +35,81 @@ namespace hkv {
 
 namespace {
 
+// ---- shared memory map of the decode kernel ----
+constexpr int kRingBytes = kDecWarps * kDecStages * kStageBytes;     // staging rings of the warps
+constexpr int kParkStride = kHeadDim + 4;                            // floats per parked output row
+constexpr int kPartOff = kRingBytes;                                 // CTA partial: acc[16][128] f32, (m, l)[16]
+constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8 + 128;
+constexpr int kSelOff = kPartOff + kPartBytes;                       // uint16 ids of the selected chunks
+constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 chunk scores
+constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers
+constexpr int kSmemBytes = kBarsOff + kDecWarps * kDecStages * 8;
+static_assert(kSmemBytes <= 232448, "decode kernel shared memory");
+static_assert(kDecStages * kStageBytes >= 16 * kParkStride * 4 + 128, "parking area fits a ring");
+static_assert(kPartOff % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0, "alignment");
+
 __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
   int i = 0;
   while (i + 1 < n && x >= prefix[i + 1]) ++i;
   return i;
 }
 
-// ---------------------------------------------------------------------------------------------
-// Chunk score + top-k (one CTA per dynamic unit).
-// score_c = <sum_g q_g, mean_c> in float32; the k_sel best chunks, ties to the lower id, are written
-// in ascending id order; n_valid = tokens those chunks hold (the last chunk of a sequence may be
-// short, and being the highest id it is always last in the list).
-// ---------------------------------------------------------------------------------------------
-constexpr int kSelThreads = 256;
-constexpr int kSelSmemScores = 8192;
+template <int NT>   // 8-wide column tiles of query heads: 1 for groups up to 8, 2 for groups up to 16
+__global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_constant__ DecodeParams P) {
+  extern __shared__ __align__(1024) uint8_t smem[];
 
-__global__ void __launch_bounds__(kSelThreads) select_chunks_kernel(const __grid_constant__ DecodeBatch batch) {
-  __shared__ float qsum[kHeadDim];
-  __shared__ float sc_smem[kSelSmemScores];
-  __shared__ int hist[256];
-  __shared__ int wsum[96];
-  __shared__ int bc[4];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int csize = P.cluster;
+  const bool clustered = csize > 1;
+  const uint32_t crank = clustered ? cluster_ctarank() : 0u;
+  // "this CTA is running": has to be known before anybody touches its shared memory remotely
+  if (clustered) cluster_arrive();
+  bool start_waited = !clustered;
 
-  const int li = find_slot(batch.dyn_prefix, batch.n, blockIdx.x);
-  char* base = batch.cache[li];
-  const Header* hdr = reinterpret_cast<const Header*>(base);
-  const int uid = reinterpret_cast<const int32_t*>(base + hdr->dyn_list_off)[blockIdx.x - batch.dyn_prefix[li]];
-  const Unit* u = reinterpret_cast<const Unit*>(base + hdr->units_off) + uid;
-  const int G = hdr->group, cs = hdr->chunk_size;
-  const int n_chunks = u->n_chunks, k_sel = u->k_sel, C = u->C;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cid = blockIdx.x / csize;
+  const int li = find_slot(P.unit_prefix, P.n, cid);
+  const int uid = cid - P.unit_prefix[li];
+  char* base = P.cache[li];
+  const Unit* up = reinterpret_cast<const Unit*>(base + kUnitsOff) + uid;
+  const int G = P.group, Hq = P.n_q_heads, cs = P.chunk_size;
+  const int ub = uid / P.n_kv_heads, uh = uid - ub * P.n_kv_heads;
+  const bool do_select = (P.phase & kPhaseSelect) != 0, do_attend = (P.phase & kPhaseAttend) != 0;
 
-  if (tid < kHeadDim) {
-    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(batch.q[li]) +
-                             (static_cast<size_t>(u->b) * hdr->n_q_heads + static_cast<size_t>(u->h) * G) * kHeadDim;
-    float s = 0.f;
-    for (int g = 0; g < G; ++g) s += __bfloat162float(q[g * kHeadDim + tid]);
-    qsum[tid] = s;
+  // the unit's record (uniform loads, issued together)
+  const int utype = up->type, C = up->C, n_tok = up->n_tok, n_chunks = up->n_chunks, k_sel = up->k_sel;
+  const uint8_t* kplane = reinterpret_cast<const uint8_t*>(base + up->k_off);
+  const uint8_t* vplane = reinterpret_cast<const uint8_t*>(base + up->v_off);
+  const uint8_t* summ = reinterpret_cast<const uint8_t*>(base + up->summ_off);
+  int32_t* gsel = reinterpret_cast<int32_t*>(base + up->idx_off);
+  float* gscores = reinterpret_cast<float*>(base + up->scores_off);
+  int32_t* n_valid_g = reinterpret_cast<int32_t*>(base + P.n_valid_off[li]) + uid;
+  int32_t* err = reinterpret_cast<int32_t*>(base + P.err_off[li]);
+  const bool dynamic = utype != 0;
+
+  if (!dynamic && !do_attend) {   // nothing to select for a static unit
+    if (clustered) cluster_wait();
+    return;
   }
-  __syncthreads();
 
-  float* scores = reinterpret_cast<float*>(base + u->scores_off);
-  const uint4* summ = reinterpret_cast<const uint4*>(base + u->summ_off);   // 16 uint4 per chunk mean
-  const bool in_smem = n_chunks <= kSelSmemScores;
+  // the group's queries as B fragments of  S^T = X Q^T  (columns >= G are zero)
+  uint32_t qb[8][2 * NT];
   {
-    // 16 lanes per chunk mean (16 B each), two chunks per warp pass
-    const int sub = lane & 15, half = lane >> 4;
-    float qv[8];
+    const uint32_t* q = reinterpret_cast<const uint32_t*>(P.q[li]) +
+                        (static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G) * (kHeadDim / 2);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) qv[j] = qsum[sub * 8 + j];
-    for (int c0 = warp * 2; c0 < n_chunks; c0 += (kSelThreads / 32) * 2) {
-      const int c = c0 + half;
-      float acc = 0.f;
-      if (c < n_chunks) {
-        const uint4 m = summ[static_cast<size_t>(c) * 16 + sub];
-        acc = fmaf(bf16_lo(m.x), qv[0], acc); acc = fmaf(bf16_hi(m.x), qv[1], acc);
-        acc = fmaf(bf16_lo(m.y), qv[2], acc); acc = fmaf(bf16_hi(m.y), qv[3], acc);
-        acc = fmaf(bf16_lo(m.z), qv[4], acc); acc = fmaf(bf16_hi(m.z), qv[5], acc);
-        acc = fmaf(bf16_lo(m.w), qv[6], acc); acc = fmaf(bf16_hi(m.w), qv[7], acc);
-      }
+    for (int nt = 0; nt < NT; ++nt) {
+      const int head = nt * 8 + g;
 #pragma unroll
-      for (int off = 8; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-      if (c < n_chunks && sub == 0) {
-        scores[c] = acc;
-        if (in_smem) sc_smem[c] = acc;
+      for (int kk = 0; kk < 8; ++kk) {
+        qb[kk][2 * nt] = (head < G) ? q[head * 64 + kk * 8 + t] : 0u;
+        qb[kk][2 * nt + 1] = (head < G) ? q[head * 64 + kk * 8 + 4 + t] : 0u;
       }
     }
   }
-  __syncthreads();
-
-  int32_t* sel = reinterpret_cast<int32_t*>(base + u->idx_off);
-  const float* src = in_smem ? sc_smem : scores;
-  int emitted;
-  if (k_sel >= n_chunks) {
-    for (int i = tid; i < n_chunks; i += kSelThreads) sel[i] = i;
-    emitted = n_chunks;
-  } else {
-    emitted = block_select_emit(
-        n_chunks, k_sel, [&](int i) { return float_key(src[i]); }, [](int) { return false; }, sel, hist, wsum, bc);
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int32_t* n_valid = reinterpret_cast<int32_t*>(base + hdr->n_valid_off);
-    int nv = emitted * cs;
-    if (emitted > 0 && sel[emitted - 1] == n_chunks - 1) nv -= n_chunks * cs - C;
-    n_valid[uid] = nv;
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Split-K flash-decode.
-//
-// One CTA per split (a contiguous range of 32-token tiles of one unit's retained token list).  Each
-// of the CTA's warps is an independent consumer with its own ring of kDecStages staging buffers and
-// its own mbarriers: it takes every kDecWarps-th tile of the split, has the TMA engine copy the
-// tile's K and V rows (1-D bulk copies, one pair per chunk piece) into the ring, and runs
-//   S = Q K^T  (rows = the group's query heads padded to 16, cols = 32 tokens)  on tensor cores,
-//   online softmax in float32 (base-2 exponent),  O += P V  on tensor cores,
-// so that every loaded KV tile is shared by all query heads of the group.  K/V rows live in HBM
-// with their eight... sixteen 16-byte pieces XOR-permuted by (row & 7) (see swz()), which makes the
-// ldmatrix reads of the staged tile bank-conflict free without any copy in shared memory.
-// At the end the warps of a CTA are merged in shared memory, the CTA writes one partial
-// (m, l, O) — or the final output when the unit has a single split — and the last CTA of a unit to
-// arrive merges the unit's partials in split order (deterministic) and writes the output.
-// ---------------------------------------------------------------------------------------------
-constexpr float kLog2e = 1.4426950408889634f;
-
-struct WarpState {
-  float m0, m1, l0, l1;
-};
-
-template <bool HI>
-__global__ void __launch_bounds__(kDecWarps * 32, 1)
-    flash_decode_kernel(const __grid_constant__ DecodeBatch batch, int out_f32) {
-  extern __shared__ __align__(1024) uint8_t smem[];
-  __shared__ int s_is_last;
-
-  const int li = find_slot(batch.split_prefix, batch.n, blockIdx.x);
-  char* base = batch.cache[li];
-  const Header* hdr = reinterpret_cast<const Header*>(base);
-  const Split sp = reinterpret_cast<const Split*>(base + hdr->splits_off)[blockIdx.x - batch.split_prefix[li]];
-  const Unit* up = reinterpret_cast<const Unit*>(base + hdr->units_off) + sp.unit;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const int G = hdr->group, Hq = hdr->n_q_heads;
-  const int cs = hdr->chunk_size;
-  const bool dynamic = up->type != 0;
-  const int ub = up->b, uh = up->h, n_splits = up->n_splits;
-  const int n_valid = dynamic ? reinterpret_cast<const int32_t*>(base + hdr->n_valid_off)[sp.unit] : up->n_tok;
-  const uint8_t* kplane = reinterpret_cast<const uint8_t*>(base + up->k_off);
-  const uint8_t* vplane = reinterpret_cast<const uint8_t*>(base + up->v_off);
-  const int32_t* sel = reinterpret_cast<const int32_t*>(base + up->idx_off);
-  int32_t* err = reinterpret_cast<int32_t*>(base + hdr->err_off);
-  const float sc = hdr->scale * kLog2e;
 
   uint8_t* ring = smem + warp * (kDecStages * kStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kDecWarps * kDecStages * kStageBytes) + warp * kDecStages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarsOff) + warp * kDecStages;
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kDecStages; ++s) mbar_init(&bars[s], 1);
@@ -150,13 +117,150 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
   }
   __syncwarp();
 
-  // tiles of this warp: first, first + kDecWarps, ... below tile_end (clipped to the valid tokens)
-  const int tile_end = min(sp.tile_end, (n_valid + kTile - 1) / kTile);
-  const int first = sp.tile_begin + warp;
+  uint32_t seq = 0;     // tiles this warp has put through its ring (stage = seq % stages)
+  bool dead = false;    // a bounded wait ran out: stop issuing, keep every barrier
+  // ldmatrix lane roles: matrix index mi = lane >> 3
+  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_piece = lane >> 4;      // non-transposed A tile
+  const int v_row = (lane & 7) + (lane >> 4) * 8, v_piece = (lane >> 3) & 1;      // transposed A tile
+
+  // =============================================================================================
+  // chunk scoring + top-k selection (dynamic units)
+  // =============================================================================================
+  float* sc_smem = reinterpret_cast<float*>(smem + kScoresOff);
+  uint16_t* sel16 = reinterpret_cast<uint16_t*>(smem + kSelOff);
+  const bool identity = dynamic && k_sel >= n_chunks;          // every chunk is loaded: no list needed
+  const bool fast = n_chunks <= kSelSmemChunks;                // scores and ids fit shared memory
+  bool sel_in_smem = false;
+  int n_valid = n_tok;
+
+  if (dynamic && do_select) {
+    const int n_st = (n_chunks + kScoreTile - 1) / kScoreTile;
+    const int st_per = (n_st + csize - 1) / csize;
+    const int st_end = min(n_st, static_cast<int>(crank + 1) * st_per);
+    const int first = static_cast<int>(crank) * st_per + warp;
+    const int n_my = first < st_end ? (st_end - first + kDecWarps - 1) / kDecWarps : 0;
+
+    auto issue_s = [&](int it) {
+      const int stage = (seq + it) % kDecStages;
+      uint8_t* st = ring + stage * kStageBytes;
+      const int r0 = (first + it * kDecWarps) * kScoreTile;
+      const int r1 = min(r0 + kScoreTile, n_chunks);
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t bytes = static_cast<uint32_t>(r1 - r0) * kRowBytes;
+        mbar_arrive_expect_tx(&bars[stage], bytes);
+        bulk_g2s(st, summ + static_cast<size_t>(r0) * kRowBytes, bytes, &bars[stage]);
+      }
+    };
+    for (int it = 0; it < min(n_my, kDecStages); ++it) issue_s(it);
+
+    if (clustered) { cluster_wait(); start_waited = true; }   // every CTA of the cluster runs: pushes are safe
+    const uint32_t sc_addr = smem_u32(sc_smem);
+
+    for (int it = 0; it < n_my; ++it) {
+      const int stage = (seq + it) % kDecStages;
+      uint8_t* st = ring + stage * kStageBytes;
+      const int r0 = (first + it * kDecWarps) * kScoreTile;
+      const int nrow = min(kScoreTile, n_chunks - r0);
+      if (!mbar_wait_bounded(&bars[stage], ((seq + it) / kDecStages) & 1)) {
+        if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrScoreWait; }
+        dead = true;
+        break;
+      }
+      const uint32_t mbase = smem_u32(st);
+#pragma unroll
+      for (int mt = 0; mt < kScoreTile / 16; ++mt) {
+        if (mt * 16 < nrow) {
+          float acc[NT][4];
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+          const uint32_t rowaddr = mbase + (mt * 16 + a_row) * kRowBytes;
+          const uint32_t key = a_row & 7;     // tiles start at multiples of 64 chunks
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
+          }
+          // chunk score = sum over the group's heads of <q_g, mean_c>
+          float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) { v0 += acc[nt][0] + acc[nt][1]; v1 += acc[nt][2] + acc[nt][3]; }
+          v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+          v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
+          v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+          v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
+          const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
+          if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
+          if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
+          if (fast) {
+            for (int s = t; s < csize; s += 4) {
+              if (c0 < n_chunks) st_cluster_f32(mapa(sc_addr + c0 * 4, s), v0);
+              if (c1 < n_chunks) st_cluster_f32(mapa(sc_addr + c1 * 4, s), v1);
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (it + kDecStages < n_my) issue_s(it + kDecStages);
+    }
+    seq += n_my;
+
+    // every score of the unit is now on its way to every CTA of the cluster
+    if (!fast) __threadfence();
+    if (clustered) { cluster_arrive(); cluster_wait(); } else { __syncthreads(); }
+
+    int* hist = reinterpret_cast<int*>(smem + kPartOff);   // the partial area is idle until the merge
+    int* wsum = hist + 256;
+    int* bc = wsum + 96;
+    int emitted;
+    if (identity) {
+      if (crank == 0) for (int i = tid; i < n_chunks; i += kDecWarps * 32) gsel[i] = i;
+      emitted = n_chunks;
+    } else if (fast) {
+      emitted = block_select_emit(
+          n_chunks, k_sel, [&](int i) { return float_key(sc_smem[i]); }, [](int) { return false; },
+          [&](int pos, int i) {
+            sel16[pos] = static_cast<uint16_t>(i);
+            if (crank == 0) gsel[pos] = i;
+          },
+          hist, wsum, bc);
+      sel_in_smem = true;
+    } else {
+      // every CTA of the cluster writes the same list to the same place
+      emitted = block_select_emit(
+          n_chunks, k_sel, [&](int i) { return float_key(__ldcg(&gscores[i])); }, [](int) { return false; },
+          [&](int pos, int i) { gsel[pos] = i; }, hist, wsum, bc);
+    }
+    __syncthreads();
+    n_valid = emitted * cs;
+    if (emitted > 0) {
+      const int last = identity ? n_chunks - 1 : (sel_in_smem ? static_cast<int>(sel16[emitted - 1]) : gsel[emitted - 1]);
+      if (last == n_chunks - 1) n_valid -= n_chunks * cs - C;   // the sequence's last chunk may be short
+    }
+    if (crank == 0 && tid == 0) *n_valid_g = n_valid;
+    if (!do_attend) return;
+  } else if (dynamic) {
+    n_valid = __ldcg(n_valid_g);   // attention only: the list of an earlier selection
+  }
+
+  // =============================================================================================
+  // flash-decoding over the unit's token list
+  // =============================================================================================
+  const bool contiguous = !dynamic || identity;
+  const float sc = P.scale_log2e;
+  const int n_tiles = (n_valid + kTile - 1) / kTile;
+  const int t_per = (n_tiles + csize - 1) / csize;
+  const int tile_end = min(n_tiles, static_cast<int>(crank + 1) * t_per);
+  const int first = static_cast<int>(crank) * t_per + warp;
   const int n_my = first < tile_end ? (tile_end - first + kDecWarps - 1) / kDecWarps : 0;
 
+  auto sel_at = [&](int i) -> int { return sel_in_smem ? static_cast<int>(sel16[i]) : gsel[i]; };
+
   auto issue = [&](int it) {
-    const int stage = it % kDecStages;
+    const int stage = (seq + it) % kDecStages;
     uint8_t* st = ring + stage * kStageBytes;
     const int v0 = (first + it * kDecWarps) * kTile;
     const int v1 = min(v0 + kTile, n_valid);
@@ -164,11 +268,11 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
     fence_proxy_async();
     if (lane == 0) mbar_arrive_expect_tx(&bars[stage], static_cast<uint32_t>(v1 - v0) * 2u * kRowBytes);
     __syncwarp();
-    if (dynamic) {
+    if (!contiguous) {
       const int ci = v0 / cs + lane;                       // lane-th chunk touching this tile
       const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
       if (p0 < p1) {
-        const size_t row = static_cast<size_t>(sel[ci]) * cs + (p0 - ci * cs);
+        const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
         const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
         bulk_g2s(st + (p0 - v0) * kRowBytes, kplane + row * kRowBytes, bytes, &bars[stage]);
         bulk_g2s(st + kTile * kRowBytes + (p0 - v0) * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
@@ -177,7 +281,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
       uint32_t key = lane & 7;
       if (v < v1) {
         const int cj = v / cs;
-        key = static_cast<uint32_t>(sel[cj] * cs + (v - cj * cs)) & 7u;
+        key = static_cast<uint32_t>(sel_at(cj) * cs + (v - cj * cs)) & 7u;
       }
       keys[lane] = key;
     } else {
@@ -190,48 +294,31 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
     }
   };
 
-  // prologue: fill the ring, then fetch this group's queries as A fragments (rows >= G are zero)
-  for (int it = 0; it < min(n_my, kDecStages); ++it) issue(it);
-
-  uint32_t qa[8][4];
-  {
-    const uint32_t* q = reinterpret_cast<const uint32_t*>(batch.q[li]) +
-                        (static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G) * (kHeadDim / 2);
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      qa[kk][0] = (g < G) ? q[g * 64 + kk * 8 + t] : 0u;
-      qa[kk][2] = (g < G) ? q[g * 64 + kk * 8 + 4 + t] : 0u;
-      if (HI) {
-        qa[kk][1] = (g + 8 < G) ? q[(g + 8) * 64 + kk * 8 + t] : 0u;
-        qa[kk][3] = (g + 8 < G) ? q[(g + 8) * 64 + kk * 8 + 4 + t] : 0u;
-      } else {
-        qa[kk][1] = 0u;
-        qa[kk][3] = 0u;
-      }
-    }
+  if (!dead) {
+    for (int it = 0; it < min(n_my, kDecStages); ++it) issue(it);
   }
 
-  float o[16][4];
+  float o[8][NT][4];
 #pragma unroll
-  for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  bool dead = false;
+  for (int dt = 0; dt < 8; ++dt) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) o[dt][nt][0] = o[dt][nt][1] = o[dt][nt][2] = o[dt][nt][3] = 0.f;
+  }
+  float mrun[NT][2], lrun[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) { mrun[nt][0] = mrun[nt][1] = -INFINITY; lrun[nt][0] = lrun[nt][1] = 0.f; }
 
-  // per-lane row roles for the two ldmatrix patterns
-  const int mj = lane >> 3, mi = lane & 7;
-  const int krow = mi + ((mj >> 1) << 3), kcsel = mj & 1;     // K (B of S = Q K^T): tokens x d-pieces
-  const int vrow = mi + ((mj & 1) << 3), vcsel = mj >> 1;     // V (B of O = P V), transposed load
-
-  for (int it = 0; it < n_my; ++it) {
-    const int stage = it % kDecStages;
+  for (int it = 0; it < n_my && !dead; ++it) {
+    const int stage = (seq + it) % kDecStages;
     uint8_t* st = ring + stage * kStageBytes;
     const int v0 = (first + it * kDecWarps) * kTile;
     const int nrow = min(kTile, n_valid - v0);
-    if (!mbar_wait_bounded(&bars[stage], (it / kDecStages) & 1)) {
+    if (!mbar_wait_bounded(&bars[stage], ((seq + it) / kDecStages) & 1)) {
       if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrDecodeWait; }
       dead = true;
       break;
     }
+    __syncwarp();   // the row keys below were written by other lanes
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(st + 2 * kTile * kRowBytes);
     if (nrow < kTile) {
       // rows past the end were not copied: clear them so that stale bits cannot poison P*V
@@ -243,86 +330,82 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
     }
     const uint32_t kbase = smem_u32(st), vbase = kbase + kTile * kRowBytes;
 
-    float s[4][4];
+    // S^T = K Q^T : rows = tokens (two 16-row tiles), columns = query heads
+    float s[2][NT][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+    for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-    for (int sl = 0; sl < 2; ++sl) {
-      const int r = sl * 16 + krow;
+      for (int nt = 0; nt < NT; ++nt) s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
+      const int r = mt * 16 + a_row;
       const uint32_t key = keys[r];
       const uint32_t rowaddr = kbase + r * kRowBytes;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(b0, b1, b2, b3, rowaddr + (((2 * kk + kcsel) ^ key) << 4));
-        mma_bf16(s[2 * sl], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
-        mma_bf16(s[2 * sl + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+        uint32_t a0, a1, a2, a3;
+        ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(s[mt][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
       }
     }
 
-    // online softmax over the tile (rows g and, for large groups, g + 8)
-    float mx0 = -INFINITY, mx1 = -INFINITY;
+    // online softmax per query head (this thread: heads 2t, 2t+1 of each column tile; tokens g, g+8 of each row tile)
+    uint32_t pb[2][NT][2];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int nt = 0; nt < NT; ++nt) {
+      float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const bool ok = (j * 8 + 2 * t + e) < nrow;
-        s[j][e] = ok ? s[j][e] * sc : -INFINITY;
-        mx0 = fmaxf(mx0, s[j][e]);
-        if (HI) {
-          s[j][2 + e] = ok ? s[j][2 + e] * sc : -INFINITY;
-          mx1 = fmaxf(mx1, s[j][2 + e]);
-        }
+      for (int mt = 0; mt < 2; ++mt) {
+        const bool ok0 = (mt * 16 + g) < nrow, ok1 = (mt * 16 + g + 8) < nrow;
+        s[mt][nt][0] = ok0 ? s[mt][nt][0] * sc : -INFINITY;
+        s[mt][nt][1] = ok0 ? s[mt][nt][1] * sc : -INFINITY;
+        s[mt][nt][2] = ok1 ? s[mt][nt][2] * sc : -INFINITY;
+        s[mt][nt][3] = ok1 ? s[mt][nt][3] * sc : -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(s[mt][nt][0], s[mt][nt][2]));
+        mx1 = fmaxf(mx1, fmaxf(s[mt][nt][1], s[mt][nt][3]));
       }
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    const float mn0 = fmaxf(m0, mx0);
-    const float c0 = exp2f(m0 - mn0);
-    m0 = mn0;
-    float c1 = 1.f;
-    if (HI) {
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float mn1 = fmaxf(m1, mx1);
-      c1 = exp2f(m1 - mn1);
-      m1 = mn1;
-    }
-    float ps0 = 0.f, ps1 = 0.f;
-    uint32_t pa[2][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float p0 = exp2f(s[j][0] - m0), p1 = exp2f(s[j][1] - m0);
-      ps0 += p0 + p1;
-      pa[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
-      if (HI) {
-        const float p2 = exp2f(s[j][2] - m1), p3 = exp2f(s[j][3] - m1);
-        ps1 += p2 + p3;
-        pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
-      } else {
-        pa[j >> 1][(j & 1) * 2 + 1] = 0u;
+      for (int off = 4; off <= 16; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
       }
-    }
-    l0 = l0 * c0 + ps0;
-    if (HI) l1 = l1 * c1 + ps1;
+      const float mn0 = fmaxf(mrun[nt][0], mx0), mn1 = fmaxf(mrun[nt][1], mx1);
+      const float c0 = exp2f(mrun[nt][0] - mn0), c1 = exp2f(mrun[nt][1] - mn1);
+      mrun[nt][0] = mn0;
+      mrun[nt][1] = mn1;
+      float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
-    for (int n = 0; n < 16; ++n) {
-      o[n][0] *= c0;
-      o[n][1] *= c0;
-      if (HI) { o[n][2] *= c1; o[n][3] *= c1; }
+      for (int mt = 0; mt < 2; ++mt) {
+        const float p0 = exp2f(s[mt][nt][0] - mn0), p1 = exp2f(s[mt][nt][1] - mn1);
+        const float p2 = exp2f(s[mt][nt][2] - mn0), p3 = exp2f(s[mt][nt][3] - mn1);
+        ps0 += p0 + p2;
+        ps1 += p1 + p3;
+        // P^T as the B operand of O^T += V^T P^T: tokens along k, heads along n
+        pb[mt][nt][0] = movmatrix_trans(pack_bf16(p0, p1));
+        pb[mt][nt][1] = movmatrix_trans(pack_bf16(p2, p3));
+      }
+      lrun[nt][0] = lrun[nt][0] * c0 + ps0;
+      lrun[nt][1] = lrun[nt][1] * c1 + ps1;
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        o[dt][nt][0] *= c0;
+        o[dt][nt][1] *= c1;
+        o[dt][nt][2] *= c0;
+        o[dt][nt][3] *= c1;
+      }
     }
 
+    // O^T += V^T P^T : rows = head-dim (eight 16-row tiles), k = tokens (two 16-token steps)
 #pragma unroll
-    for (int sl = 0; sl < 2; ++sl) {
-      const int r = sl * 16 + vrow;
+    for (int ks = 0; ks < 2; ++ks) {
+      const int r = ks * 16 + v_row;
       const uint32_t key = keys[r];
       const uint32_t rowaddr = vbase + r * kRowBytes;
 #pragma unroll
-      for (int np = 0; np < 8; ++np) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_trans(b0, b1, b2, b3, rowaddr + (((2 * np + vcsel) ^ key) << 4));
-        mma_bf16(o[2 * np], pa[sl][0], pa[sl][1], pa[sl][2], pa[sl][3], b0, b1);
-        mma_bf16(o[2 * np + 1], pa[sl][0], pa[sl][1], pa[sl][2], pa[sl][3], b2, b3);
+      for (int dt = 0; dt < 8; ++dt) {
+        uint32_t a0, a1, a2, a3;
+        ldsm_x4_trans(a0, a1, a2, a3, rowaddr + (((2 * dt + v_piece) ^ key) << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(o[dt][nt], a0, a1, a2, a3, pb[ks][nt][0], pb[ks][nt][1]);
       }
     }
     __syncwarp();
@@ -337,121 +420,170 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1)
   }
 
   // ---- merge the warps of this CTA ----
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-  if (HI) {
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  }
-  // each warp parks (m, l, O) in its own (now idle) ring: [16][128] floats, then m[16], l[16]
+  // each warp parks (m, l, O) in its own (now idle) ring: O as [16 heads][kParkStride] floats, then m[16], l[16]
   float* wo = reinterpret_cast<float*>(ring);
-  float* wm = wo + 16 * kHeadDim;
+  float* wm = wo + 16 * kParkStride;
   float* wl = wm + 16;
 #pragma unroll
-  for (int n = 0; n < 16; ++n) {
-    *reinterpret_cast<float2*>(&wo[g * kHeadDim + n * 8 + 2 * t]) = make_float2(o[n][0], o[n][1]);
-    if (HI) *reinterpret_cast<float2*>(&wo[(g + 8) * kHeadDim + n * 8 + 2 * t]) = make_float2(o[n][2], o[n][3]);
-  }
-  if (t == 0) {
-    wm[g] = m0; wl[g] = l0;
-    wm[g + 8] = HI ? m1 : -INFINITY;
-    wl[g + 8] = HI ? l1 : 0.f;
+  for (int nt = 0; nt < NT; ++nt) {
+    float l0 = lrun[nt][0], l1 = lrun[nt][1];
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
+    const int h0 = nt * 8 + 2 * t;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) {
+      wo[h0 * kParkStride + dt * 16 + g] = o[dt][nt][0];
+      wo[(h0 + 1) * kParkStride + dt * 16 + g] = o[dt][nt][1];
+      wo[h0 * kParkStride + dt * 16 + g + 8] = o[dt][nt][2];
+      wo[(h0 + 1) * kParkStride + dt * 16 + g + 8] = o[dt][nt][3];
+    }
+    if (g == 0) {
+      wm[h0] = mrun[nt][0]; wm[h0 + 1] = mrun[nt][1];
+      wl[h0] = l0; wl[h0 + 1] = l1;
+    }
   }
   __syncthreads();
 
-  const int d = threadIdx.x;   // blockDim.x == kHeadDim
-  const size_t pstride = static_cast<size_t>(G) * (kHeadDim + 2);
-  float* partials = reinterpret_cast<float*>(base + hdr->partials_off);
-  float* mypart = partials + (static_cast<size_t>(up->split_base) + sp.slot) * pstride;
+  const int d = tid;   // blockDim.x == kHeadDim
   const size_t out_row0 = static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G;
+  float* part = reinterpret_cast<float*>(smem + kPartOff);
+  float2* part_ml = reinterpret_cast<float2*>(smem + kPartOff + kMaxGroup * kHeadDim * 4);
+  auto store_out = [&](int row, float r) {
+    if (P.out_f32) reinterpret_cast<float*>(P.out[li])[(out_row0 + row) * kHeadDim + d] = r;
+    else reinterpret_cast<__nv_bfloat16*>(P.out[li])[(out_row0 + row) * kHeadDim + d] = __float2bfloat16_rn(r);
+  };
   for (int row = 0; row < G; ++row) {
     float M = -INFINITY;
 #pragma unroll
     for (int w2 = 0; w2 < kDecWarps; ++w2)
-      M = fmaxf(M, reinterpret_cast<const float*>(smem + w2 * (kDecStages * kStageBytes))[16 * kHeadDim + row]);
+      M = fmaxf(M, reinterpret_cast<const float*>(smem + w2 * (kDecStages * kStageBytes))[16 * kParkStride + row]);
     float acc = 0.f, L = 0.f;
     if (M > -INFINITY) {
 #pragma unroll
       for (int w2 = 0; w2 < kDecWarps; ++w2) {
         const float* po = reinterpret_cast<const float*>(smem + w2 * (kDecStages * kStageBytes));
-        const float f = exp2f(po[16 * kHeadDim + row] - M);
-        acc += po[row * kHeadDim + d] * f;
-        L += po[16 * kHeadDim + 16 + row] * f;
+        const float f = exp2f(po[16 * kParkStride + row] - M);
+        acc += po[row * kParkStride + d] * f;
+        L += po[16 * kParkStride + 16 + row] * f;
       }
     }
-    if (n_splits == 1) {
-      const float r = (L > 0.f && !dead) ? acc / L : 0.f;
-      if (out_f32) reinterpret_cast<float*>(batch.out[li])[(out_row0 + row) * kHeadDim + d] = r;
-      else reinterpret_cast<__nv_bfloat16*>(batch.out[li])[(out_row0 + row) * kHeadDim + d] = __float2bfloat16_rn(r);
+    if (!clustered) {
+      store_out(row, L > 0.f ? acc / L : 0.f);
     } else {
-      mypart[row * kHeadDim + d] = acc;
-      if (d == 0) { mypart[G * kHeadDim + row] = M; mypart[G * kHeadDim + G + row] = L; }
+      part[row * kHeadDim + d] = acc;
+      if (d == 0) part_ml[row] = make_float2(M, L);
     }
   }
-  if (n_splits == 1) return;
+  if (!clustered) return;
 
-  // ---- the last split of the unit to arrive merges all of them, in split order ----
-  int32_t* counter = reinterpret_cast<int32_t*>(base + hdr->counters_off) + sp.unit;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int prev = atomicAdd(counter, 1);
-    s_is_last = (prev == n_splits - 1);
-  }
-  __syncthreads();
-  if (!s_is_last) return;
-  __threadfence();
-  const float* up_part = partials + static_cast<size_t>(up->split_base) * pstride;
-  for (int row = 0; row < G; ++row) {
+  // ---- merge the CTAs of the cluster through distributed shared memory ----
+  if (!start_waited) cluster_wait();
+  cluster_arrive();
+  cluster_wait();
+  const uint32_t part_addr = smem_u32(part), ml_addr = smem_u32(part_ml);
+  for (int row = static_cast<int>(crank); row < G; row += csize) {
+    float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
+#pragma unroll
+    for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+      if (s2 < csize) {
+        const float2 ml = ld_cluster_f32x2(mapa(ml_addr + row * 8, s2));
+        ms[s2] = ml.x;
+        ls[s2] = ml.y;
+        av[s2] = ld_cluster_f32(mapa(part_addr + (row * kHeadDim + d) * 4, s2));
+      } else {
+        ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f;
+      }
+    }
     float M = -INFINITY;
-    for (int s2 = 0; s2 < n_splits; ++s2) M = fmaxf(M, __ldcg(&up_part[s2 * pstride + G * kHeadDim + row]));
+#pragma unroll
+    for (int s2 = 0; s2 < kMaxCluster; ++s2) M = fmaxf(M, ms[s2]);
     float acc = 0.f, L = 0.f;
     if (M > -INFINITY) {
-      for (int s2 = 0; s2 < n_splits; ++s2) {
-        const float* p = up_part + s2 * pstride;
-        const float f = exp2f(__ldcg(&p[G * kHeadDim + row]) - M);
-        acc += __ldcg(&p[row * kHeadDim + d]) * f;
-        L += __ldcg(&p[G * kHeadDim + G + row]) * f;
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+        const float f = exp2f(ms[s2] - M);
+        acc += av[s2] * f;
+        L += ls[s2] * f;
       }
     }
-    const float r = L > 0.f ? acc / L : 0.f;
-    if (out_f32) reinterpret_cast<float*>(batch.out[li])[(out_row0 + row) * kHeadDim + d] = r;
-    else reinterpret_cast<__nv_bfloat16*>(batch.out[li])[(out_row0 + row) * kHeadDim + d] = __float2bfloat16_rn(r);
+    store_out(row, L > 0.f ? acc / L : 0.f);
   }
-  if (threadIdx.x == 0) *counter = 0;   // ready for the next step
+  // nobody leaves while its partial may still be read
+  cluster_arrive();
+  cluster_wait();
+}
+
+template <int NT>
+void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clusters, int cluster, cudaStream_t stream) {
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(static_cast<unsigned>(n_clusters) * cluster, 1, 1);
+  cfg.blockDim = dim3(kDecWarps * 32, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+}
+
+// One-time set-up of a kernel instance: shared-memory size, permission for clusters above eight
+// CTAs, and the largest cluster size the device can co-schedule with this footprint.
+template <int NT>
+cudaError_t configure(int* max_cluster) {
+  static int cached = 0;
+  if (cached == 0) {
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    int best = 1;
+    for (int c = kMaxCluster; c > 1; c >>= 1) {
+      cudaLaunchConfig_t cfg;
+      cudaLaunchAttribute attr[1];
+      fill_config<NT>(cfg, attr, 1, c, nullptr);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<NT>, &cfg) == cudaSuccess && n >= 1) { best = c; break; }
+      cudaGetLastError();
+    }
+    cached = best;
+  }
+  *max_cluster = cached;
+  return cudaSuccess;
+}
+
+template <int NT>
+cudaError_t launch_nt(const DecodeParams& params, int total_units, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fill_config<NT>(cfg, attr, total_units, params.cluster, stream);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<NT>, params);
 }
 
 }  // namespace
 
-size_t flash_decode_smem_bytes() {
-  return static_cast<size_t>(kDecWarps) * kDecStages * kStageBytes + kDecWarps * kDecStages * sizeof(uint64_t);
+size_t decode_smem_bytes() { return kSmemBytes; }
+
+int choose_cluster(int total_units, int max_tiles, int sm_count) {
+  // the largest power of two that keeps the launch within one wave of CTAs (one CTA per SM) and
+  // leaves every CTA at least two tiles of the longest unit
+  int c = 1;
+  while (c * 2 <= kMaxCluster && static_cast<int64_t>(total_units) * c * 2 <= sm_count && c * 2 * 2 <= max_tiles) c *= 2;
+  return c;
 }
 
-cudaError_t launch_select_chunks(const DecodeBatch& batch, int total_dyn, cudaStream_t stream) {
-  if (total_dyn <= 0) return cudaSuccess;
-  select_chunks_kernel<<<total_dyn, kSelThreads, 0, stream>>>(batch);
-  return cudaGetLastError();
+cudaError_t decode_max_cluster(int group, int* max_cluster) {
+  return group > 8 ? configure<2>(max_cluster) : configure<1>(max_cluster);
 }
 
-cudaError_t launch_flash_decode(const DecodeBatch& batch, int total_splits, int group, bool out_f32,
-                                cudaStream_t stream) {
-  if (total_splits <= 0) return cudaSuccess;
-  const size_t smem = flash_decode_smem_bytes();
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(flash_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(flash_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  if (group > 8)
-    flash_decode_kernel<true><<<total_splits, kDecWarps * 32, smem, stream>>>(batch, out_f32 ? 1 : 0);
-  else
-    flash_decode_kernel<false><<<total_splits, kDecWarps * 32, smem, stream>>>(batch, out_f32 ? 1 : 0);
-  return cudaGetLastError();
+cudaError_t launch_decode(const DecodeParams& params, int total_units, cudaStream_t stream) {
+  if (total_units <= 0) return cudaSuccess;
+  if (params.group > 8) return launch_nt<2>(params, total_units, stream);
+  return launch_nt<1>(params, total_units, stream);
 }
 
 }  // namespace hkv

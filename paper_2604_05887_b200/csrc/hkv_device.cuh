@@ -85,6 +85,46 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
+// transposes an 8x8 matrix of 16-bit elements held in the usual fragment layout (thread 4g+t owns
+// row g, columns 2t and 2t+1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+// ---- thread-block cluster: rank, barrier, distributed shared memory ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// address of the same shared-memory location in the CTA of rank `rank` of this cluster
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
 // ---- order-preserving key of a finite float: larger float <=> larger key; every key > 0 ----
 __device__ __forceinline__ uint32_t float_key(float f) {
   f = f + 0.0f;   // -0 -> +0 so that equal floats have equal keys
@@ -95,12 +135,13 @@ __device__ __forceinline__ uint32_t float_key(float f) {
 // ---------------------------------------------------------------------------------------------
 // Block-wide exact selection.  Among the n items, every item with always(i) is emitted, and of the
 // items with key(i) != 0 ("candidates") the k with the largest keys are emitted, equal keys going
-// to the lower index.  Emission is in ascending index order into out[]; returns the number emitted
-// (valid in every thread).  Requires k <= number of candidates, blockDim.x a multiple of 32 and at
-// most 1024.  hist: 256 ints, wsum: 3*32 ints, bc: 4 ints of shared memory.
+// to the lower index.  Emission is in ascending index order: emit(position, index) is called once
+// per selected item; returns the number emitted (valid in every thread).  Requires k <= number of
+// candidates, blockDim.x a multiple of 32 and at most 1024.  hist: 256 ints, wsum: 3*32 ints,
+// bc: 4 ints of shared memory.
 // ---------------------------------------------------------------------------------------------
-template <class KeyFn, class AlwaysFn>
-__device__ int block_select_emit(int n, int k, KeyFn key, AlwaysFn always, int32_t* out, int* hist, int* wsum,
+template <class KeyFn, class AlwaysFn, class EmitFn>
+__device__ int block_select_emit(int n, int k, KeyFn key, AlwaysFn always, EmitFn emit, int* hist, int* wsum,
                                  int* bc) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   uint32_t prefix = 0, mask = 0;
@@ -176,7 +217,7 @@ __device__ int block_select_emit(int n, int k, KeyFn key, AlwaysFn always, int32
       if (w2 < warp) sel_before += c;
       sel_total += c;
     }
-    if (sel) out[sel_before + __popc(bsel & ((1u << lane) - 1u))] = i;
+    if (sel) emit(sel_before + __popc(bsel & ((1u << lane) - 1u)), i);
     emitted += sel_total;
     eq_seen += eq_total;
     __syncthreads();
