@@ -186,6 +186,7 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
       st = HKV_ERR_WORKSPACE;
     if (st != HKV_OK) { delete c; return st; }
     c->dev_base = static_cast<char*>(cache_mem);
+    c->fresh = true;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const Header& H = c->hdr;
 
@@ -231,6 +232,8 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   for (int i = 0; i < n; ++i) {
     const hkv_cache* c = caches[i];
     if (!c || !q[i] || (do_attend && !out[i])) return HKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q[i]) & 3) || (do_attend && (reinterpret_cast<uintptr_t>(out[i]) & 15)))
+      return HKV_ERR_INVALID_ARG;
     const Header& H = c->hdr;
     const Header& H0 = caches[0]->hdr;
     if (H.group != H0.group || H.n_q_heads != H0.n_q_heads || H.n_kv_heads != H0.n_kv_heads ||
@@ -251,14 +254,21 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   P.scale_log2e = H0.scale * 1.4426950408889634f;
   P.phase = (do_select ? kPhaseSelect : 0u) | (do_attend ? kPhaseAttend : 0u);
   P.out_f32 = (H0.flags & HKV_OUT_F32) ? 1u : 0u;
-  int max_cluster = 1;
-  if (decode_max_cluster(P.group, &max_cluster) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  const int* max_active = nullptr;
+  if (decode_cluster_caps(P.group, &max_active) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
   const int total_units = P.unit_prefix[n];
-  P.cluster = std::min(max_cluster, choose_cluster(total_units, max_tiles, sm_count()));
+  P.cluster = choose_cluster(total_units, max_tiles, max_active);
+  // The launch may overlap the tail of a preceding decode launch (it touches nothing that depends on
+  // earlier work before its dependency wait).  Right after hkv_compress the cache itself is what
+  // the preceding kernels are still writing, so that first launch is fully serialised.
+  bool fresh = false;
+  for (int i = 0; i < n; ++i) fresh = fresh || caches[i]->fresh;
+  P.pdl = fresh ? 0u : 1u;
   if (launch_decode(P, total_units, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
     cudaGetLastError();
     return HKV_ERR_CUDA;
   }
+  for (int i = 0; i < n; ++i) caches[i]->fresh = false;
   return HKV_OK;
 }
 
@@ -377,7 +387,17 @@ hkv_status hkv_cache_stats(const hkv_cache* c, hkv_stats* st) {
   st->workspace_bytes = static_cast<int64_t>(c->workspace_bytes);
   st->n_static = c->hdr.n_static;
   st->n_dynamic = c->hdr.n_dynamic;
-  st->n_splits = c->hdr.n_units * choose_cluster(c->hdr.n_units, c->max_tiles, sm_count());
+  {
+    // CTAs of a decode launch on this cache alone; without a device, the capacities of a B200
+    const int* max_active = nullptr;
+    int assumed[kMaxCluster + 1] = {};
+    if (decode_cluster_caps(c->hdr.group, &max_active) != cudaSuccess) {
+      cudaGetLastError();
+      for (int k = 1; k <= kMaxCluster; k <<= 1) assumed[k] = 2 * 148 / k;
+      max_active = assumed;
+    }
+    st->n_splits = c->hdr.n_units * choose_cluster(c->hdr.n_units, c->max_tiles, max_active);
+  }
   st->launches_per_decode = 1;
   return HKV_OK;
 }

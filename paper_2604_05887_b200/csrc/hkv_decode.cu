@@ -2,12 +2,18 @@
 // selection (dynamic heads), flash-decoding over the unit's retained token list, and the merge of
 // the partial results — one launch per layer.
 //
-// Work decomposition.  A thread-block CLUSTER of `cluster` CTAs owns one unit.  Inside a CTA every
-// warp is an independent consumer with its own ring of kDecStages staging buffers and its own
-// mbarriers; the TMA engine fills the ring with 1-D bulk copies (no multicast).
+// Work decomposition.  A thread-block CLUSTER of `cluster` CTAs owns one unit.  A CTA has a ring of
+// kDecStages staging buffers filled by the TMA engine with 1-D bulk copies (no multicast), each
+// completing on its own mbarrier; tile j of the CTA lives in stage j % kDecStages and is consumed by
+// warp j % kDecWarps, which then re-arms the stage with tile j + kDecStages.  Because the warp that
+// arms a stage is not the warp that consumes it, a consumer first checks the stage's "armed with
+// tile" counter and only then waits on the mbarrier's phase parity (parity alone cannot tell a
+// phase from the one two later, and a fast warp may get that far ahead).  The footprint is kept
+// under half an SM's shared memory so that two CTAs — of this launch or of two consecutive
+// launches — are resident per SM.
 //
 //   dynamic unit, selection:  the cluster's CTAs split the unit's chunk means between them; a warp
-//     stages 64 means at a time and computes  S^T = M Q^T  (rows = chunks, columns = the group's
+//     takes up to 64 staged means and computes  S^T = M Q^T  (rows = chunks, columns = the group's
 //     query heads) on tensor cores; the chunk score is the float32 sum over the group's heads.
 //     Scores are pushed into the shared memory of every CTA of the cluster (distributed shared
 //     memory), a cluster barrier follows, and each CTA then runs the same exact radix selection on
@@ -15,13 +21,18 @@
 //     round trip through global memory.
 //   every unit, attention:  the unit's token list (static: the compacted rows; dynamic: the rows of
 //     the selected chunks) is cut into 32-token tiles, dealt to the cluster's CTAs as contiguous
-//     ranges and to a CTA's warps round-robin.  Per tile:  S^T = K Q^T  (rows = tokens, columns =
-//     query heads, so the group shares every loaded KV tile and no tensor-core row is padding),
-//     online softmax in float32 (base-2 exponent), P^T moved into operand layout with movmatrix,
-//     O^T += V^T P^T.
+//     ranges.  Per tile:  S^T = K Q^T  (rows = tokens, columns = query heads, so the group shares
+//     every loaded KV tile and no tensor-core row is padding), online softmax in float32 (base-2
+//     exponent), P^T moved into operand layout with movmatrix,  O^T += V^T P^T.
 //   merge:  the warps of a CTA are combined in shared memory; the CTAs of the cluster read each
-//     other's partial (m, l, O) through distributed shared memory, CTA r producing output rows
-//     r, r + cluster, ... — fixed order, no atomics, deterministic.
+//     other's partial (m, l, O) through distributed shared memory, each producing a slice of the
+//     output — fixed order, no atomics, deterministic.
+//
+// Programmatic dependent launch.  Nothing the kernel does before griddepcontrol.wait depends on the
+// step's query or on an earlier decode launch: it reads the unit table, arms the barriers and has
+// the first ring-full of K/V rows (or chunk means) copied in.  A launch that follows another decode
+// launch on the stream may therefore start while its predecessor is still running; it reads q and
+// writes anything only after the wait.
 //
 // K/V rows and chunk means live in HBM with their sixteen 16-byte pieces XOR-permuted by (row & 7),
 // which makes the ldmatrix reads of a staged tile bank-conflict free without any copy in shared
@@ -36,16 +47,18 @@ namespace hkv {
 namespace {
 
 // ---- shared memory map of the decode kernel ----
-constexpr int kRingBytes = kDecWarps * kDecStages * kStageBytes;     // staging rings of the warps
+constexpr int kRingBytes = kDecStages * kStageBytes;                 // staging ring
 constexpr int kParkStride = kHeadDim + 4;                            // floats per parked output row
-constexpr int kPartOff = kRingBytes;                                 // CTA partial: acc[16][128] f32, (m, l)[16]
-constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8 + 128;
-constexpr int kSelOff = kPartOff + kPartBytes;                       // uint16 ids of the selected chunks
+constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp's (O, m, l)
+constexpr int kPartOff = kDecWarps * kParkBytes;                     // CTA partial: acc[16][128] f32, (m, l)[16]
+constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
+constexpr int kSelOff = kRingBytes;                                  // uint16 ids of the selected chunks
 constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 chunk scores
 constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers
-constexpr int kSmemBytes = kBarsOff + kDecWarps * kDecStages * 8;
-static_assert(kSmemBytes <= 232448, "decode kernel shared memory");
-static_assert(kDecStages * kStageBytes >= 16 * kParkStride * 4 + 128, "parking area fits a ring");
+constexpr int kArmedOff = kBarsOff + kDecStages * 8;                 // per stage: sequence number of the tile it was last armed with
+constexpr int kSmemBytes = kArmedOff + kDecStages * 4 + 8;
+static_assert(kDecCtasPerSm * (kSmemBytes + 1024) <= 233472, "two CTAs per SM");
+static_assert(kPartOff + kPartBytes <= kRingBytes, "parking and the CTA partial reuse the idle ring");
 static_assert(kPartOff % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0, "alignment");
 
 __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
@@ -54,8 +67,23 @@ __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
   return i;
 }
 
+// Checked build (-DHKV_CHECKED): every index that feeds an address is validated first; a violation is
+// recorded in the cache's error word (HKV_ERR_INDEX, detail = place) and the access is skipped.
+#ifdef HKV_CHECKED
+#define HKV_CHECK(cond, place)                                             \
+  if (!(cond)) {                                                           \
+    if (atomicCAS(&err[0], 0, HKV_ERR_INDEX) == 0) err[1] = (place);       \
+    dead = true;                                                           \
+  }
+#else
+#define HKV_CHECK(cond, place)
+#endif
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <int NT>   // 8-wide column tiles of query heads: 1 for groups up to 8, 2 for groups up to 16
-__global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_constant__ DecodeParams P) {
+__global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(const __grid_constant__ DecodeParams P) {
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -63,6 +91,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
   const int csize = P.cluster;
   const bool clustered = csize > 1;
   const uint32_t crank = clustered ? cluster_ctarank() : 0u;
+  pdl_launch_dependents();
   // "this CTA is running": has to be known before anybody touches its shared memory remotely
   if (clustered) cluster_arrive();
   bool start_waited = !clustered;
@@ -78,6 +107,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
 
   // the unit's record (uniform loads, issued together)
   const int utype = up->type, C = up->C, n_tok = up->n_tok, n_chunks = up->n_chunks, k_sel = up->k_sel;
+#ifdef HKV_CHECKED
+  const int plane_rows = up->plane_rows;
+#endif
   const uint8_t* kplane = reinterpret_cast<const uint8_t*>(base + up->k_off);
   const uint8_t* vplane = reinterpret_cast<const uint8_t*>(base + up->v_off);
   const uint8_t* summ = reinterpret_cast<const uint8_t*>(base + up->summ_off);
@@ -92,6 +124,142 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
     return;
   }
 
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarsOff);
+  volatile uint32_t* armed = reinterpret_cast<volatile uint32_t*>(smem + kArmedOff);
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kDecStages; ++s) { mbar_init(&bars[s], 1); armed[s] = 0u; }
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  // Waits until stage `stage` holds the tile with ring sequence number `q` (0-based over both
+  // phases): first until it has been armed with that tile, then until the copies have landed.
+  // Both waits are bounded; false = gave up.
+  auto wait_tile = [&](int stage, uint32_t q) -> bool {
+    if (armed[stage] != q + 1u) {
+      const long long start = clock64();
+      for (uint32_t it = 1; armed[stage] != q + 1u; ++it) {
+        if ((it & 255u) == 0u && clock64() - start > 2000000000ll) return false;
+      }
+    }
+    return mbar_wait_bounded(&bars[stage], (q / kDecStages) & 1u);
+  };
+
+  bool dead = false;    // a bounded wait ran out: stop issuing, keep every barrier
+  // ldmatrix lane roles: matrix index mi = lane >> 3
+  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_piece = lane >> 4;      // non-transposed A tile
+  const int v_row = (lane & 7) + (lane >> 4) * 8, v_piece = (lane >> 3) & 1;      // transposed A tile
+
+  float* sc_smem = reinterpret_cast<float*>(smem + kScoresOff);
+  uint16_t* sel16 = reinterpret_cast<uint16_t*>(smem + kSelOff);
+  const bool identity = dynamic && k_sel >= n_chunks;          // every chunk is loaded: no list needed
+  const bool fast = n_chunks <= kSelSmemChunks;                // scores and ids fit shared memory
+  const bool contiguous = !dynamic || identity;
+  const bool scoring = dynamic && do_select;
+  bool sel_in_smem = false;
+  uint32_t seq0 = 0;    // tiles the CTA's ring has carried in earlier phases
+
+  // ---- attention phase: tiles [at_tile0, at_tile0 + at_n) of the unit's token list ----
+  int n_valid = 0, at_tile0 = 0, at_n = 0;
+  auto setup_attn = [&](int nv) {
+    n_valid = nv;
+    const int n_tiles = (nv + kTile - 1) / kTile;
+    const int t_per = (n_tiles + csize - 1) / csize;
+    at_tile0 = static_cast<int>(crank) * t_per;
+    at_n = max(0, min(n_tiles, at_tile0 + t_per) - at_tile0);
+  };
+  auto sel_at = [&](int i) -> int { return sel_in_smem ? static_cast<int>(sel16[i]) : gsel[i]; };
+  auto issue_attn = [&](int j) {   // whole warp; arms stage (seq0 + j) % stages with CTA tile j
+    const int stage = (seq0 + j) % kDecStages;
+    uint8_t* st = smem + stage * kStageBytes;
+    const int v0 = (at_tile0 + j) * kTile;
+    const int v1 = min(v0 + kTile, n_valid);
+    uint32_t* keys = reinterpret_cast<uint32_t*>(st + 2 * kTile * kRowBytes);
+    int ci = 0, p0 = 0, p1 = 0;
+    if (!contiguous) {
+      ci = v0 / cs + lane;                                 // lane-th chunk touching this tile
+      p0 = max(v0, ci * cs);
+      p1 = min(v1, (ci + 1) * cs);
+      const int v = v0 + lane;
+      uint32_t key = lane & 7;
+      if (v < v1) {
+        const int cj = v / cs;
+        key = static_cast<uint32_t>(sel_at(cj) * cs + (v - cj * cs)) & 7u;
+      }
+      keys[lane] = key;
+    } else {
+      keys[lane] = lane & 7;
+    }
+    HKV_CHECK(v0 >= 0 && v0 < v1 && v1 - v0 <= kTile, 100);
+    HKV_CHECK(contiguous ? (v1 <= plane_rows) : true, 101);
+#ifdef HKV_CHECKED
+    if (!contiguous && p0 < p1) {
+      const int sid = sel_at(ci);
+      HKV_CHECK(sid >= 0 && sid < n_chunks, 102);
+      HKV_CHECK(static_cast<int64_t>(sid) * cs + (p0 - ci * cs) + (p1 - p0) <= plane_rows, 103);
+      HKV_CHECK(p0 - v0 >= 0 && p1 - v0 <= kTile, 104);
+    }
+    dead = __any_sync(0xffffffffu, dead);
+    if (dead) return;
+#endif
+    __syncwarp();
+    if (lane == 0) {
+      armed[stage] = seq0 + static_cast<uint32_t>(j) + 1u;
+      mbar_arrive_expect_tx(&bars[stage], static_cast<uint32_t>(v1 - v0) * 2u * kRowBytes);
+    }
+    __syncwarp();
+    if (!contiguous) {
+      if (p0 < p1) {
+        const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
+        const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
+        bulk_g2s(st + (p0 - v0) * kRowBytes, kplane + row * kRowBytes, bytes, &bars[stage]);
+        bulk_g2s(st + kTile * kRowBytes + (p0 - v0) * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
+      }
+    } else if (lane == 0) {
+      const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
+      bulk_g2s(st, kplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
+      bulk_g2s(st + kTile * kRowBytes, vplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
+    }
+  };
+
+  // ---- scoring phase: tiles of sc_rows chunk means, [sc_tile0, sc_tile0 + sc_n) for this CTA ----
+  int sc_rows = 16, sc_tile0 = 0, sc_n = 0;
+  if (scoring) {
+    const int per_cta = (n_chunks + csize - 1) / csize;
+    sc_rows = per_cta >= 4 * kScoreTile ? kScoreTile : (per_cta >= 2 * kScoreTile ? kScoreTile / 2 : 16);
+    const int n_st = (n_chunks + sc_rows - 1) / sc_rows;
+    const int st_per = (n_st + csize - 1) / csize;
+    sc_tile0 = static_cast<int>(crank) * st_per;
+    sc_n = max(0, min(n_st, sc_tile0 + st_per) - sc_tile0);
+  }
+  auto issue_score = [&](int j) {
+    if (lane == 0) {
+      const int stage = j % kDecStages;
+      const int r0 = (sc_tile0 + j) * sc_rows;
+      const uint32_t bytes = static_cast<uint32_t>(min(r0 + sc_rows, n_chunks) - r0) * kRowBytes;
+      HKV_CHECK(r0 >= 0 && r0 < n_chunks && bytes <= 2u * kTile * kRowBytes, 120);
+#ifdef HKV_CHECKED
+      if (dead) return;
+#endif
+      armed[stage] = static_cast<uint32_t>(j) + 1u;
+      mbar_arrive_expect_tx(&bars[stage], bytes);
+      bulk_g2s(smem + stage * kStageBytes, summ + static_cast<size_t>(r0) * kRowBytes, bytes, &bars[stage]);
+    }
+  };
+
+  // ---- copies that do not depend on this step's query start before the dependency wait ----
+  bool attn_armed = false;
+  if (scoring) {
+    for (int j = warp; j < min(sc_n, kDecStages); j += kDecWarps) issue_score(j);
+  } else if (!dynamic) {
+    setup_attn(n_tok);
+    for (int j = warp; j < min(at_n, kDecStages); j += kDecWarps) issue_attn(j);
+    attn_armed = true;
+  }
+
+  pdl_wait();
+
   // the group's queries as B fragments of  S^T = X Q^T  (columns >= G are zero)
   uint32_t qb[8][2 * NT];
   {
@@ -102,117 +270,78 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
       const int head = nt * 8 + g;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
-        qb[kk][2 * nt] = (head < G) ? q[head * 64 + kk * 8 + t] : 0u;
-        qb[kk][2 * nt + 1] = (head < G) ? q[head * 64 + kk * 8 + 4 + t] : 0u;
+        qb[kk][2 * nt] = (head < G) ? __ldg(&q[head * 64 + kk * 8 + t]) : 0u;
+        qb[kk][2 * nt + 1] = (head < G) ? __ldg(&q[head * 64 + kk * 8 + 4 + t]) : 0u;
       }
     }
   }
-
-  uint8_t* ring = smem + warp * (kDecStages * kStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarsOff) + warp * kDecStages;
-  if (lane == 0) {
-#pragma unroll
-    for (int s = 0; s < kDecStages; ++s) mbar_init(&bars[s], 1);
-    mbar_fence_init();
-  }
-  __syncwarp();
-
-  uint32_t seq = 0;     // tiles this warp has put through its ring (stage = seq % stages)
-  bool dead = false;    // a bounded wait ran out: stop issuing, keep every barrier
-  // ldmatrix lane roles: matrix index mi = lane >> 3
-  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_piece = lane >> 4;      // non-transposed A tile
-  const int v_row = (lane & 7) + (lane >> 4) * 8, v_piece = (lane >> 3) & 1;      // transposed A tile
 
   // =============================================================================================
   // chunk scoring + top-k selection (dynamic units)
   // =============================================================================================
-  float* sc_smem = reinterpret_cast<float*>(smem + kScoresOff);
-  uint16_t* sel16 = reinterpret_cast<uint16_t*>(smem + kSelOff);
-  const bool identity = dynamic && k_sel >= n_chunks;          // every chunk is loaded: no list needed
-  const bool fast = n_chunks <= kSelSmemChunks;                // scores and ids fit shared memory
-  bool sel_in_smem = false;
-  int n_valid = n_tok;
-
-  if (dynamic && do_select) {
-    const int n_st = (n_chunks + kScoreTile - 1) / kScoreTile;
-    const int st_per = (n_st + csize - 1) / csize;
-    const int st_end = min(n_st, static_cast<int>(crank + 1) * st_per);
-    const int first = static_cast<int>(crank) * st_per + warp;
-    const int n_my = first < st_end ? (st_end - first + kDecWarps - 1) / kDecWarps : 0;
-
-    auto issue_s = [&](int it) {
-      const int stage = (seq + it) % kDecStages;
-      uint8_t* st = ring + stage * kStageBytes;
-      const int r0 = (first + it * kDecWarps) * kScoreTile;
-      const int r1 = min(r0 + kScoreTile, n_chunks);
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t bytes = static_cast<uint32_t>(r1 - r0) * kRowBytes;
-        mbar_arrive_expect_tx(&bars[stage], bytes);
-        bulk_g2s(st, summ + static_cast<size_t>(r0) * kRowBytes, bytes, &bars[stage]);
-      }
-    };
-    for (int it = 0; it < min(n_my, kDecStages); ++it) issue_s(it);
-
+  if (scoring) {
     if (clustered) { cluster_wait(); start_waited = true; }   // every CTA of the cluster runs: pushes are safe
     const uint32_t sc_addr = smem_u32(sc_smem);
+    const int n_mt = sc_rows >> 4;
 
-    for (int it = 0; it < n_my; ++it) {
-      const int stage = (seq + it) % kDecStages;
-      uint8_t* st = ring + stage * kStageBytes;
-      const int r0 = (first + it * kDecWarps) * kScoreTile;
-      const int nrow = min(kScoreTile, n_chunks - r0);
-      if (!mbar_wait_bounded(&bars[stage], ((seq + it) / kDecStages) & 1)) {
+    for (int j = warp; j < sc_n; j += kDecWarps) {
+      const int stage = j % kDecStages;
+      const int r0 = (sc_tile0 + j) * sc_rows;
+      const int nrow = min(sc_rows, n_chunks - r0);
+      if (!wait_tile(stage, static_cast<uint32_t>(j))) {
         if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrScoreWait; }
         dead = true;
         break;
       }
-      const uint32_t mbase = smem_u32(st);
+      const uint32_t mbase = smem_u32(smem + stage * kStageBytes);
+      for (int mt = 0; mt < n_mt; ++mt) {
+        if (mt * 16 >= nrow) break;
+        float acc[2][NT][4];
 #pragma unroll
-      for (int mt = 0; mt < kScoreTile / 16; ++mt) {
-        if (mt * 16 < nrow) {
-          float acc[NT][4];
+        for (int e = 0; e < 2; ++e) {
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-          const uint32_t rowaddr = mbase + (mt * 16 + a_row) * kRowBytes;
-          const uint32_t key = a_row & 7;     // tiles start at multiples of 64 chunks
+          for (int nt = 0; nt < NT; ++nt) acc[e][nt][0] = acc[e][nt][1] = acc[e][nt][2] = acc[e][nt][3] = 0.f;
+        }
+        const uint32_t rowaddr = mbase + (mt * 16 + a_row) * kRowBytes;
+        const uint32_t key = a_row & 7;     // tiles start at multiples of 16 chunks
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            uint32_t a0, a1, a2, a3;
-            ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
+        for (int kk = 0; kk < 8; ++kk) {
+          uint32_t a0, a1, a2, a3;
+          ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
-          }
-          // chunk score = sum over the group's heads of <q_g, mean_c>
-          float v0 = 0.f, v1 = 0.f;
+          for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[kk & 1][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
+        }
+        // chunk score = sum over the group's heads of <q_g, mean_c>
+        float v0 = 0.f, v1 = 0.f;
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) { v0 += acc[nt][0] + acc[nt][1]; v1 += acc[nt][2] + acc[nt][3]; }
-          v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
-          v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
-          v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-          v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
-          const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
-          if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
-          if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
-          if (fast) {
-            for (int s = t; s < csize; s += 4) {
-              if (c0 < n_chunks) st_cluster_f32(mapa(sc_addr + c0 * 4, s), v0);
-              if (c1 < n_chunks) st_cluster_f32(mapa(sc_addr + c1 * 4, s), v1);
-            }
+        for (int nt = 0; nt < NT; ++nt) {
+          v0 += (acc[0][nt][0] + acc[1][nt][0]) + (acc[0][nt][1] + acc[1][nt][1]);
+          v1 += (acc[0][nt][2] + acc[1][nt][2]) + (acc[0][nt][3] + acc[1][nt][3]);
+        }
+        v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+        v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
+        const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
+        if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
+        if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
+        if (fast) {
+          for (int s = t; s < csize; s += 4) {
+            if (c0 < n_chunks) st_cluster_f32(mapa(sc_addr + c0 * 4, s), v0);
+            if (c1 < n_chunks) st_cluster_f32(mapa(sc_addr + c1 * 4, s), v1);
           }
         }
       }
       __syncwarp();
-      if (it + kDecStages < n_my) issue_s(it + kDecStages);
+      if (j + kDecStages < sc_n) issue_score(j + kDecStages);
     }
-    seq += n_my;
+    seq0 = static_cast<uint32_t>(sc_n);
 
     // every score of the unit is now on its way to every CTA of the cluster
     if (!fast) __threadfence();
     if (clustered) { cluster_arrive(); cluster_wait(); } else { __syncthreads(); }
 
-    int* hist = reinterpret_cast<int*>(smem + kPartOff);   // the partial area is idle until the merge
+    int* hist = reinterpret_cast<int*>(smem);   // the ring is idle between the two phases
     int* wsum = hist + 256;
     int* bc = wsum + 96;
     int emitted;
@@ -235,67 +364,25 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
           [&](int pos, int i) { gsel[pos] = i; }, hist, wsum, bc);
     }
     __syncthreads();
-    n_valid = emitted * cs;
+    fence_proxy_async();   // the selection's scratch in the ring is about to be overwritten by bulk copies
+    int nv = emitted * cs;
     if (emitted > 0) {
       const int last = identity ? n_chunks - 1 : (sel_in_smem ? static_cast<int>(sel16[emitted - 1]) : gsel[emitted - 1]);
-      if (last == n_chunks - 1) n_valid -= n_chunks * cs - C;   // the sequence's last chunk may be short
+      if (last == n_chunks - 1) nv -= n_chunks * cs - C;   // the sequence's last chunk may be short
     }
-    if (crank == 0 && tid == 0) *n_valid_g = n_valid;
+    if (crank == 0 && tid == 0) *n_valid_g = nv;
     if (!do_attend) return;
+    setup_attn(nv);
   } else if (dynamic) {
-    n_valid = __ldcg(n_valid_g);   // attention only: the list of an earlier selection
+    setup_attn(__ldcg(n_valid_g));   // attention only: the list of an earlier selection
   }
 
   // =============================================================================================
   // flash-decoding over the unit's token list
   // =============================================================================================
-  const bool contiguous = !dynamic || identity;
   const float sc = P.scale_log2e;
-  const int n_tiles = (n_valid + kTile - 1) / kTile;
-  const int t_per = (n_tiles + csize - 1) / csize;
-  const int tile_end = min(n_tiles, static_cast<int>(crank + 1) * t_per);
-  const int first = static_cast<int>(crank) * t_per + warp;
-  const int n_my = first < tile_end ? (tile_end - first + kDecWarps - 1) / kDecWarps : 0;
-
-  auto sel_at = [&](int i) -> int { return sel_in_smem ? static_cast<int>(sel16[i]) : gsel[i]; };
-
-  auto issue = [&](int it) {
-    const int stage = (seq + it) % kDecStages;
-    uint8_t* st = ring + stage * kStageBytes;
-    const int v0 = (first + it * kDecWarps) * kTile;
-    const int v1 = min(v0 + kTile, n_valid);
-    uint32_t* keys = reinterpret_cast<uint32_t*>(st + 2 * kTile * kRowBytes);
-    fence_proxy_async();
-    if (lane == 0) mbar_arrive_expect_tx(&bars[stage], static_cast<uint32_t>(v1 - v0) * 2u * kRowBytes);
-    __syncwarp();
-    if (!contiguous) {
-      const int ci = v0 / cs + lane;                       // lane-th chunk touching this tile
-      const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
-      if (p0 < p1) {
-        const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
-        const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
-        bulk_g2s(st + (p0 - v0) * kRowBytes, kplane + row * kRowBytes, bytes, &bars[stage]);
-        bulk_g2s(st + kTile * kRowBytes + (p0 - v0) * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
-      }
-      const int v = v0 + lane;
-      uint32_t key = lane & 7;
-      if (v < v1) {
-        const int cj = v / cs;
-        key = static_cast<uint32_t>(sel_at(cj) * cs + (v - cj * cs)) & 7u;
-      }
-      keys[lane] = key;
-    } else {
-      if (lane == 0) {
-        const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
-        bulk_g2s(st, kplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
-        bulk_g2s(st + kTile * kRowBytes, vplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
-      }
-      keys[lane] = lane & 7;
-    }
-  };
-
-  if (!dead) {
-    for (int it = 0; it < min(n_my, kDecStages); ++it) issue(it);
+  if (!attn_armed && !dead) {
+    for (int j = warp; j < min(at_n, kDecStages); j += kDecWarps) issue_attn(j);
   }
 
   float o[8][NT][4];
@@ -308,34 +395,45 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) { mrun[nt][0] = mrun[nt][1] = -INFINITY; lrun[nt][0] = lrun[nt][1] = 0.f; }
 
-  for (int it = 0; it < n_my && !dead; ++it) {
-    const int stage = (seq + it) % kDecStages;
-    uint8_t* st = ring + stage * kStageBytes;
-    const int v0 = (first + it * kDecWarps) * kTile;
+  for (int j = warp; j < at_n && !dead; j += kDecWarps) {
+    const int stage = (seq0 + j) % kDecStages;
+    uint8_t* st = smem + stage * kStageBytes;
+    const int v0 = (at_tile0 + j) * kTile;
     const int nrow = min(kTile, n_valid - v0);
-    if (!mbar_wait_bounded(&bars[stage], ((seq + it) / kDecStages) & 1)) {
+    if (!wait_tile(stage, seq0 + static_cast<uint32_t>(j))) {
       if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrDecodeWait; }
       dead = true;
       break;
     }
-    __syncwarp();   // the row keys below were written by other lanes
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(st + 2 * kTile * kRowBytes);
+#ifdef HKV_CHECKED
+    HKV_CHECK(keys[lane] < 8u, 110);
+    HKV_CHECK(nrow >= 1, 111);
+    dead = __any_sync(0xffffffffu, dead);
+    if (dead) break;
+#endif
     if (nrow < kTile) {
       // rows past the end were not copied: clear them so that stale bits cannot poison P*V
       for (int r = nrow; r < kTile; ++r) {
         reinterpret_cast<uint2*>(st + r * kRowBytes)[lane] = make_uint2(0u, 0u);
         reinterpret_cast<uint2*>(st + kTile * kRowBytes + r * kRowBytes)[lane] = make_uint2(0u, 0u);
       }
+      fence_proxy_async();
       __syncwarp();
     }
     const uint32_t kbase = smem_u32(st), vbase = kbase + kTile * kRowBytes;
 
-    // S^T = K Q^T : rows = tokens (two 16-row tiles), columns = query heads
+    // S^T = K Q^T : rows = tokens (two 16-row tiles), columns = query heads; the reduction over the
+    // head dimension runs as two interleaved accumulation chains
     float s[2][NT][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
+      float s2[NT][4];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
+      for (int nt = 0; nt < NT; ++nt) {
+        s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
+        s2[nt][0] = s2[nt][1] = s2[nt][2] = s2[nt][3] = 0.f;
+      }
       const int r = mt * 16 + a_row;
       const uint32_t key = keys[r];
       const uint32_t rowaddr = kbase + r * kRowBytes;
@@ -344,7 +442,15 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
         uint32_t a0, a1, a2, a3;
         ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) mma_bf16(s[mt][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
+        for (int nt = 0; nt < NT; ++nt) {
+          if (kk & 1) mma_bf16(s2[nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
+          else mma_bf16(s[mt][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
+        }
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        s[mt][nt][0] += s2[nt][0]; s[mt][nt][1] += s2[nt][1];
+        s[mt][nt][2] += s2[nt][2]; s[mt][nt][3] += s2[nt][3];
       }
     }
 
@@ -409,72 +515,89 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
       }
     }
     __syncwarp();
-    if (it + kDecStages < n_my) issue(it + kDecStages);
+    if (j + kDecStages < at_n) issue_attn(j + kDecStages);
   }
 
-  if (dead) {
-    // leave only after our own copies in flight had another bounded chance to land
+  // a warp that gave up tells the others, so that nobody parks results over copies still in flight
+  if (__syncthreads_or(dead ? 1 : 0)) {
+    // leave only after every armed stage had another bounded chance to receive its copies
     for (int s2 = 0; s2 < kDecStages; ++s2) {
-      for (int it = 0; it < 1024 && !mbar_try_wait(&bars[s2], 0) && !mbar_try_wait(&bars[s2], 1); ++it) {}
+      const uint32_t a = armed[s2];
+      if (a != 0u) mbar_wait_bounded(&bars[s2], ((a - 1u) / kDecStages) & 1u);
     }
+    __syncthreads();
   }
+  // the ring is idle from here on: it now holds the partial results
 
   // ---- merge the warps of this CTA ----
-  // each warp parks (m, l, O) in its own (now idle) ring: O as [16 heads][kParkStride] floats, then m[16], l[16]
-  float* wo = reinterpret_cast<float*>(ring);
-  float* wm = wo + 16 * kParkStride;
-  float* wl = wm + 16;
+  // each warp parks (m, l, O): O as [16 heads][kParkStride] floats, then m[16], l[16]
+  {
+    float* wo = reinterpret_cast<float*>(smem + warp * kParkBytes);
+    float* wm = wo + 16 * kParkStride;
+    float* wl = wm + 16;
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    float l0 = lrun[nt][0], l1 = lrun[nt][1];
+    for (int nt = 0; nt < NT; ++nt) {
+      float l0 = lrun[nt][0], l1 = lrun[nt][1];
 #pragma unroll
-    for (int off = 4; off <= 16; off <<= 1) {
-      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-    }
-    const int h0 = nt * 8 + 2 * t;
+      for (int off = 4; off <= 16; off <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+      }
+      const int h0 = nt * 8 + 2 * t;
 #pragma unroll
-    for (int dt = 0; dt < 8; ++dt) {
-      wo[h0 * kParkStride + dt * 16 + g] = o[dt][nt][0];
-      wo[(h0 + 1) * kParkStride + dt * 16 + g] = o[dt][nt][1];
-      wo[h0 * kParkStride + dt * 16 + g + 8] = o[dt][nt][2];
-      wo[(h0 + 1) * kParkStride + dt * 16 + g + 8] = o[dt][nt][3];
-    }
-    if (g == 0) {
-      wm[h0] = mrun[nt][0]; wm[h0 + 1] = mrun[nt][1];
-      wl[h0] = l0; wl[h0 + 1] = l1;
+      for (int dt = 0; dt < 8; ++dt) {
+        wo[h0 * kParkStride + dt * 16 + g] = o[dt][nt][0];
+        wo[(h0 + 1) * kParkStride + dt * 16 + g] = o[dt][nt][1];
+        wo[h0 * kParkStride + dt * 16 + g + 8] = o[dt][nt][2];
+        wo[(h0 + 1) * kParkStride + dt * 16 + g + 8] = o[dt][nt][3];
+      }
+      if (g == 0) {
+        wm[h0] = mrun[nt][0]; wm[h0 + 1] = mrun[nt][1];
+        wl[h0] = l0; wl[h0 + 1] = l1;
+      }
     }
   }
   __syncthreads();
 
-  const int d = tid;   // blockDim.x == kHeadDim
   const size_t out_row0 = static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G;
   float* part = reinterpret_cast<float*>(smem + kPartOff);
   float2* part_ml = reinterpret_cast<float2*>(smem + kPartOff + kMaxGroup * kHeadDim * 4);
-  auto store_out = [&](int row, float r) {
-    if (P.out_f32) reinterpret_cast<float*>(P.out[li])[(out_row0 + row) * kHeadDim + d] = r;
-    else reinterpret_cast<__nv_bfloat16*>(P.out[li])[(out_row0 + row) * kHeadDim + d] = __float2bfloat16_rn(r);
-  };
-  for (int row = 0; row < G; ++row) {
-    float M = -INFINITY;
+  // items = (row, group of four columns): independent loads, one pass for groups up to 4, two up to 8
+  for (int item = tid; item < G * 32; item += kDecWarps * 32) {
+    const int row = item >> 5, dq = item & 31;
+    float mw[kDecWarps], M = -INFINITY;
 #pragma unroll
-    for (int w2 = 0; w2 < kDecWarps; ++w2)
-      M = fmaxf(M, reinterpret_cast<const float*>(smem + w2 * (kDecStages * kStageBytes))[16 * kParkStride + row]);
-    float acc = 0.f, L = 0.f;
+    for (int w2 = 0; w2 < kDecWarps; ++w2) {
+      mw[w2] = reinterpret_cast<const float*>(smem + w2 * kParkBytes)[16 * kParkStride + row];
+      M = fmaxf(M, mw[w2]);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
     if (M > -INFINITY) {
 #pragma unroll
       for (int w2 = 0; w2 < kDecWarps; ++w2) {
-        const float* po = reinterpret_cast<const float*>(smem + w2 * (kDecStages * kStageBytes));
-        const float f = exp2f(po[16 * kParkStride + row] - M);
-        acc += po[row * kParkStride + d] * f;
+        const float* po = reinterpret_cast<const float*>(smem + w2 * kParkBytes);
+        const float f = exp2f(mw[w2] - M);
+        const float4 v = *reinterpret_cast<const float4*>(po + row * kParkStride + dq * 4);
+        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
         L += po[16 * kParkStride + 16 + row] * f;
       }
     }
     if (!clustered) {
-      store_out(row, L > 0.f ? acc / L : 0.f);
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+      const size_t off = (out_row0 + row) * kHeadDim + dq * 4;
+      if (P.out_f32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(P.out[li]) + off) =
+            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+      } else {
+        uint2 pk;
+        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(P.out[li]) + off) = pk;
+      }
     } else {
-      part[row * kHeadDim + d] = acc;
-      if (d == 0) part_ml[row] = make_float2(M, L);
+      *reinterpret_cast<float4*>(part + row * kHeadDim + dq * 4) = acc;
+      if (dq == 0) part_ml[row] = make_float2(M, L);
     }
   }
   if (!clustered) return;
@@ -483,33 +606,42 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
   if (!start_waited) cluster_wait();
   cluster_arrive();
   cluster_wait();
-  const uint32_t part_addr = smem_u32(part), ml_addr = smem_u32(part_ml);
-  for (int row = static_cast<int>(crank); row < G; row += csize) {
-    float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
-#pragma unroll
-    for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-      if (s2 < csize) {
-        const float2 ml = ld_cluster_f32x2(mapa(ml_addr + row * 8, s2));
-        ms[s2] = ml.x;
-        ls[s2] = ml.y;
-        av[s2] = ld_cluster_f32(mapa(part_addr + (row * kHeadDim + d) * 4, s2));
-      } else {
-        ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f;
-      }
-    }
-    float M = -INFINITY;
-#pragma unroll
-    for (int s2 = 0; s2 < kMaxCluster; ++s2) M = fmaxf(M, ms[s2]);
-    float acc = 0.f, L = 0.f;
-    if (M > -INFINITY) {
+  {
+    const uint32_t part_addr = smem_u32(part), ml_addr = smem_u32(part_ml);
+    const int total = G * kHeadDim;
+    const int per = (total + csize - 1) / csize;
+    const int e_end = min(total, static_cast<int>(crank + 1) * per);
+    for (int e = static_cast<int>(crank) * per + tid; e < e_end; e += kDecWarps * 32) {
+      const int row = e >> 7;
+      float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
 #pragma unroll
       for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-        const float f = exp2f(ms[s2] - M);
-        acc += av[s2] * f;
-        L += ls[s2] * f;
+        if (s2 < csize) {
+          const float2 ml = ld_cluster_f32x2(mapa(ml_addr + row * 8, s2));
+          ms[s2] = ml.x;
+          ls[s2] = ml.y;
+          av[s2] = ld_cluster_f32(mapa(part_addr + e * 4, s2));
+        } else {
+          ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f;
+        }
       }
+      float M = -INFINITY;
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) M = fmaxf(M, ms[s2]);
+      float acc = 0.f, L = 0.f;
+      if (M > -INFINITY) {
+#pragma unroll
+        for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+          const float f = exp2f(ms[s2] - M);
+          acc += av[s2] * f;
+          L += ls[s2] * f;
+        }
+      }
+      const float r = L > 0.f ? acc / L : 0.f;
+      const size_t off = out_row0 * kHeadDim + e;
+      if (P.out_f32) reinterpret_cast<float*>(P.out[li])[off] = r;
+      else reinterpret_cast<__nv_bfloat16*>(P.out[li])[off] = __float2bfloat16_rn(r);
     }
-    store_out(row, L > 0.f ? acc / L : 0.f);
   }
   // nobody leaves while its partial may still be read
   cluster_arrive();
@@ -517,7 +649,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(const __grid_
 }
 
 template <int NT>
-void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clusters, int cluster, cudaStream_t stream) {
+void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clusters, int cluster, bool pdl,
+                 cudaStream_t stream) {
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(static_cast<unsigned>(n_clusters) * cluster, 1, 1);
   cfg.blockDim = dim3(kDecWarps * 32, 1, 1);
@@ -527,40 +660,49 @@ void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clust
   attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (pdl) {
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
 }
 
 // One-time set-up of a kernel instance: shared-memory size, permission for clusters above eight
-// CTAs, and the largest cluster size the device can co-schedule with this footprint.
+// CTAs, and for every cluster size how many clusters the device can hold at once.
+struct ClusterCaps {
+  bool ready = false;
+  int max_active[kMaxCluster + 1] = {};
+};
+
 template <int NT>
-cudaError_t configure(int* max_cluster) {
-  static int cached = 0;
-  if (cached == 0) {
+cudaError_t configure(const ClusterCaps** out) {
+  static ClusterCaps caps;
+  if (!caps.ready) {
     cudaError_t e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
-    int best = 1;
-    for (int c = kMaxCluster; c > 1; c >>= 1) {
+    for (int c = 1; c <= kMaxCluster; c <<= 1) {
       cudaLaunchConfig_t cfg;
-      cudaLaunchAttribute attr[1];
-      fill_config<NT>(cfg, attr, 1, c, nullptr);
+      cudaLaunchAttribute attr[2];
+      fill_config<NT>(cfg, attr, 1, c, false, nullptr);
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<NT>, &cfg) == cudaSuccess && n >= 1) { best = c; break; }
-      cudaGetLastError();
+      if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<NT>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+      caps.max_active[c] = n;
     }
-    cached = best;
+    caps.ready = true;
   }
-  *max_cluster = cached;
+  *out = &caps;
   return cudaSuccess;
 }
 
 template <int NT>
 cudaError_t launch_nt(const DecodeParams& params, int total_units, cudaStream_t stream) {
   cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[1];
-  fill_config<NT>(cfg, attr, total_units, params.cluster, stream);
+  cudaLaunchAttribute attr[2];
+  fill_config<NT>(cfg, attr, total_units, params.cluster, params.pdl != 0, stream);
   return cudaLaunchKernelEx(&cfg, decode_kernel<NT>, params);
 }
 
@@ -568,16 +710,20 @@ cudaError_t launch_nt(const DecodeParams& params, int total_units, cudaStream_t 
 
 size_t decode_smem_bytes() { return kSmemBytes; }
 
-int choose_cluster(int total_units, int max_tiles, int sm_count) {
-  // the largest power of two that keeps the launch within one wave of CTAs (one CTA per SM) and
-  // leaves every CTA at least two tiles of the longest unit
+int choose_cluster(int total_units, int max_tiles, const int* max_active) {
+  // The largest power of two that (a) the device can hold in ONE wave of clusters, (b) leaves every
+  // CTA at least two tiles of the longest unit.  max_active[c] = clusters of size c resident at once.
   int c = 1;
-  while (c * 2 <= kMaxCluster && static_cast<int64_t>(total_units) * c * 2 <= sm_count && c * 2 * 2 <= max_tiles) c *= 2;
+  while (c * 2 <= kMaxCluster && max_active[c * 2] >= total_units && c * 2 * 2 <= max_tiles) c *= 2;
   return c;
 }
 
-cudaError_t decode_max_cluster(int group, int* max_cluster) {
-  return group > 8 ? configure<2>(max_cluster) : configure<1>(max_cluster);
+cudaError_t decode_cluster_caps(int group, const int** max_active) {
+  const ClusterCaps* caps = nullptr;
+  cudaError_t e = group > 8 ? configure<2>(&caps) : configure<1>(&caps);
+  if (e != cudaSuccess) return e;
+  *max_active = caps->max_active;
+  return cudaSuccess;
 }
 
 cudaError_t launch_decode(const DecodeParams& params, int total_units, cudaStream_t stream) {

@@ -18,11 +18,11 @@ constexpr int kAlign = 256;
 constexpr int kMaxCluster = 16;           // CTAs that may share one (sequence, kv head) unit
 
 // decode kernel launch shape
-constexpr int kDecWarps = 4;              // warps per CTA, each with its own staging ring
-constexpr int kDecStages = 3;             // ring depth per warp (tiles in flight)
+constexpr int kDecWarps = 4;              // consumer warps per CTA
+constexpr int kDecStages = 6;             // staging ring of a CTA (tiles in flight); two CTAs fit one SM
 constexpr int kStageBytes = kTile * kRowBytes * 2 + 128;   // K tile + V tile + row keys
-constexpr int kScoreTile = 2 * kTile;     // chunk means one stage holds while chunks are scored
-constexpr int kSelSmemChunks = 4096;      // chunk scores / selected ids a CTA keeps in shared memory
+constexpr int kScoreTile = 2 * kTile;     // most chunk means one stage holds while chunks are scored
+constexpr int kSelSmemChunks = 2048;      // chunk scores / selected ids a CTA keeps in shared memory
 
 // One (sequence b, kv head h) pair of a layer; unit id = b * n_kv_heads + h.
 struct Unit {
@@ -69,6 +69,7 @@ struct DecodeParams {
   float scale_log2e;
   uint32_t phase;      // kPhaseSelect | kPhaseAttend
   uint32_t out_f32;
+  uint32_t pdl;        // launched with programmatic stream serialization
   int32_t unit_prefix[kMaxMulti + 1];
   char* cache[kMaxMulti];
   const void* q[kMaxMulti];
@@ -80,12 +81,16 @@ struct DecodeParams {
 // device error word helpers
 enum ErrPlace : int32_t { kErrDecodeWait = 1, kErrIndex = 2, kErrScoreWait = 3 };
 
+// Upper bound on resident CTAs per SM the decode kernel is built for.
+constexpr int kDecCtasPerSm = 2;
+
 // ---- kernel launchers (definitions in the .cu files) ----
-// Picks the cluster size for `total_units` units whose longest token list has `max_tiles` tiles.
-int choose_cluster(int total_units, int max_tiles, int sm_count);
-// Largest cluster size the device co-schedules for the decode kernel of this group size (also
-// performs the kernel's one-time set-up; call before the first launch_decode).
-cudaError_t decode_max_cluster(int group, int* max_cluster);
+// Picks the cluster size for `total_units` units whose longest token list has `max_tiles` tiles;
+// max_active[c] = clusters of c CTAs the device holds at once (index 1, 2, 4, 8, 16).
+int choose_cluster(int total_units, int max_tiles, const int* max_active);
+// Cluster capacities of the decode kernel for this group size (also performs the kernel's one-time
+// set-up; call before the first launch_decode).
+cudaError_t decode_cluster_caps(int group, const int** max_active);
 cudaError_t launch_decode(const DecodeParams& params, int total_units, cudaStream_t stream);
 cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, const void* q_obs,
                                  const Header& hdr, const std::vector<Unit>& units, int64_t ws_rowstat_off,
@@ -108,4 +113,5 @@ struct hkv_cache {
   size_t cache_bytes, workspace_bytes;
   int64_t kv_bytes, summary_bytes, algo_bytes, retained;
   int max_static_rows, max_dyn_rows, max_chunks, max_tiles;
+  bool fresh;   // no decode launch has followed the compression yet
 };

@@ -110,6 +110,35 @@ def test_ragged_tail_chunk_and_many_splits(P):
     assert rep["stats"]["n_splits"] > L.batch * L.n_kv_heads
 
 
+def test_more_chunks_than_fit_shared_memory(P):
+    """chunk size 1 on a few thousand tokens: the selection works on scores and id lists in global memory."""
+    L = small(C=2600, cs=1, B=1, budget=0.3, w=16, head_type=[[1, 0, 1, 1]])
+    rep = P.compare_layer(L)
+    L = small(C=2300, cs=1, B=2, budget=1.0, w=16)          # every chunk selected: no list at all
+    P.compare_layer(L)
+
+
+def test_back_to_back_steps_overlap_safely(P):
+    """Several decode launches in a row on one stream (each may start before its predecessor has
+    finished): every step's output must still match a step run in isolation."""
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    L = hi.cfg1(layer=0, C=4096, block=512, n_steps=6)
+    lc = LayerCache(L)
+    qs = [to_device_bf16(q) for q in L.q]
+    alone = []
+    for q in qs:
+        alone.append(lc.decode(q).clone())
+        torch.cuda.synchronize()
+    outs = [lc.new_out() for _ in qs]
+    for rep in range(3):
+        for q, o_ in zip(qs, outs):
+            lc.decode(q, o_)
+    torch.cuda.synchronize()
+    for a, b in zip(alone, outs):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    lc.close()
+
+
 def test_determinism_and_static_independent_of_dynamic_budget():
     from paper_2604_05887_b200 import binding as hkv
     from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
