@@ -158,6 +158,28 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
 
 hkv_status hkv_cache_destroy(hkv_cache* cache);
 
+/* Chunk scoring + top-k for one dynamic head WITHOUT any caller- or library-allocated scratch.
+ * (The paper has no counterpart: this is a packaging variant of the selection step of
+ * hkv_select_chunks.)  It exists for callers that cannot allocate device memory where they call
+ * from — code running inside another runtime's callback or a latency-critical loop, where
+ * cudaMalloc (or a framework allocator) is forbidden or would synchronise the device.  They pass
+ * inputs and the output only; the float32 score per chunk, which the other entry points keep in
+ * cache_mem, lives in a fixed array inside the library (HKV_NOALLOC_MAX_CHUNKS floats = 256 KiB,
+ * held by every GPU that loads the library until the process exits).
+ *   q        dev bf16 [group, 128]      the query heads that share the KV head
+ *   means    dev bf16 [n_chunks, 128]   chunk means, plain row-major (16-byte aligned)
+ *   group    1..16;  n_chunks 1..HKV_NOALLOC_MAX_CHUNKS (more -> HKV_ERR_WORKSPACE);  k >= 1
+ *   out_ids  dev int32 [min(k, n_chunks)]  ids of the k highest-scoring chunks, ascending; score =
+ *            sum over the group of <q_g, mean_c> in float32, ties to the lower id
+ * Allocates nothing and never synchronises.  The first call on each device looks up the array's
+ * device address (current device = the one that will run the call); make that first call outside
+ * any stream capture.  All calls on a device share the one array and it keeps the last call's
+ * scores (every entry in use is rewritten before it is read, nothing needs clearing): two calls
+ * that overlap on the GPU, on any streams, race — serialise them. */
+#define HKV_NOALLOC_MAX_CHUNKS 65536
+hkv_status hkv_topk_chunks_noalloc(const void* q, const void* means, int32_t group, int32_t n_chunks,
+                                   int32_t k, int32_t* out_ids, void* stream);
+
 /* ---- introspection (parity tests, roofline numerator). These synchronise the given stream. ---- */
 
 /* kept positions of static head (b, h), ascending; host_out has room for `capacity` ints. */

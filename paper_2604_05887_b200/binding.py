@@ -25,7 +25,8 @@ STATUS_NAMES = {0: "HKV_OK", 1: "HKV_ERR_INVALID_ARG", 2: "HKV_ERR_SHAPE", 3: "H
 EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi", "hkv_select_chunks",
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
-           "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string"]
+           "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
+           "hkv_topk_chunks_noalloc"]
 
 
 class hkv_config(C.Structure):
@@ -74,6 +75,7 @@ def _load() -> C.CDLL:
     lib.hkv_window_scores_offset.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
     lib.hkv_cache_stats.argtypes = [vp, C.POINTER(hkv_stats)]
     lib.hkv_last_device_error.argtypes = [vp, i32p, i32p, vp]
+    lib.hkv_topk_chunks_noalloc.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
     lib.hkv_status_string.argtypes = [C.c_int]
     lib.hkv_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -178,6 +180,16 @@ def hkv_decode_attn_host(cache: int, q_host, out_host, q_dev, out_dev, stream=No
         raise ValueError("q_host and out_host must be contiguous CPU tensors")
     _check(lib.hkv_decode_attn_host(cache, q_host.data_ptr(), out_host.data_ptr(), _dev(q_dev), _dev(out_dev),
                                     _stream(stream)), "hkv_decode_attn_host")
+
+
+HKV_NOALLOC_MAX_CHUNKS = 65536
+
+
+def hkv_topk_chunks_noalloc(q, means, k: int, out_ids, stream=None) -> None:
+    """Top-k chunks of one dynamic head with the library's built-in score scratch (no allocation).
+    q: bf16 CUDA [group, 128]; means: bf16 CUDA [n_chunks, 128] plain row-major; out_ids: int32 CUDA [min(k, n_chunks)]."""
+    _check(lib.hkv_topk_chunks_noalloc(_dev(q), _dev(means), int(q.shape[0]), int(means.shape[0]), int(k),
+                                       _dev(out_ids), _stream(stream)), "hkv_topk_chunks_noalloc")
 
 
 def hkv_cache_destroy(cache: int) -> None:
