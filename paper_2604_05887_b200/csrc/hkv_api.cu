@@ -16,16 +16,6 @@ namespace {
 
 inline int64_t align_up(int64_t x, int64_t a = kAlign) { return (x + a - 1) / a * a; }
 
-int sm_count() {
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-      n <= 0) {
-    cudaGetLastError();   // clear
-    return 148;
-  }
-  return n;
-}
-
 hkv_status check_config(const hkv_config* cfg) {
   if (!cfg) return HKV_ERR_INVALID_ARG;
   if (cfg->batch < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->max_seq_len < 1) return HKV_ERR_SHAPE;
@@ -222,6 +212,19 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
   }
 }
 
+#ifdef HKV_PROFILE
+static unsigned long long* g_prof = nullptr;
+static long long g_prof_ctas = 0, g_prof_cursor = 0;
+// Profiling build only: device buffer of kProfSlots x 8 bytes per CTA; successive decode launches
+// take successive regions of it (a launch that no longer fits is not recorded).
+extern "C" int hkv_profile_attach(void* dev_buffer, long long n_ctas) {
+  g_prof = static_cast<unsigned long long*>(dev_buffer);
+  g_prof_ctas = n_ctas;
+  g_prof_cursor = 0;
+  return 0;
+}
+#endif
+
 static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, void* const* out, int32_t n,
                                 void* stream, bool do_select, bool do_attend) {
   if (!caches || !q || n < 1 || n > kMaxMulti || (do_attend && !out)) return HKV_ERR_INVALID_ARG;
@@ -264,6 +267,16 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   bool fresh = false;
   for (int i = 0; i < n; ++i) fresh = fresh || caches[i]->fresh;
   P.pdl = fresh ? 0u : 1u;
+#ifdef HKV_PROFILE
+  {
+    const long long ctas = static_cast<long long>(total_units) * P.cluster;
+    P.prof = nullptr;
+    if (g_prof && g_prof_cursor + ctas <= g_prof_ctas) {
+      P.prof = g_prof + g_prof_cursor * kProfSlots;
+      g_prof_cursor += ctas;
+    }
+  }
+#endif
   if (launch_decode(P, total_units, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
     cudaGetLastError();
     return HKV_ERR_CUDA;

@@ -5,7 +5,7 @@
 // Work decomposition.  A thread-block CLUSTER of `cluster` CTAs owns one unit.  A CTA has a ring of
 // kDecStages staging buffers filled by the TMA engine with 1-D bulk copies (no multicast), each
 // completing on its own mbarrier; tile j of the CTA lives in stage j % kDecStages and is consumed by
-// warp j % kDecWarps, which then re-arms the stage with tile j + kDecStages.  Because the warp that
+// one of the CTA's W warps (j % W), which then re-arms the stage with tile j + kDecStages.  Because the warp that
 // arms a stage is not the warp that consumes it, a consumer first checks the stage's "armed with
 // tile" counter and only then waits on the mbarrier's phase parity (parity alone cannot tell a
 // phase from the one two later, and a fast warp may get that far ahead).  The footprint is kept
@@ -50,16 +50,19 @@ namespace {
 constexpr int kRingBytes = kDecStages * kStageBytes;                 // staging ring
 constexpr int kParkStride = kHeadDim + 4;                            // floats per parked output row
 constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp's (O, m, l)
-constexpr int kPartOff = kDecWarps * kParkBytes;                     // CTA partial: acc[16][128] f32, (m, l)[16]
+constexpr int kMaxWarps = 8;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
+constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
 constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
 constexpr int kSelOff = kRingBytes;                                  // uint16 ids of the selected chunks
 constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 chunk scores
 constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers
 constexpr int kArmedOff = kBarsOff + kDecStages * 8;                 // per stage: sequence number of the tile it was last armed with
-constexpr int kSmemBytes = kArmedOff + kDecStages * 4 + 8;
+constexpr int kTopkOff = kArmedOff + kDecStages * 4 + 8;             // scratch of the selection (never touched by bulk copies)
+constexpr int kSmemBytes = kTopkOff + kTopkScratchInts * 4;
 static_assert(kDecCtasPerSm * (kSmemBytes + 1024) <= 233472, "two CTAs per SM");
-static_assert(kPartOff + kPartBytes <= kRingBytes, "parking and the CTA partial reuse the idle ring");
-static_assert(kPartOff % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0, "alignment");
+static_assert(part_off(kMaxWarps) + kPartBytes <= kRingBytes, "parking and the CTA partial reuse the idle ring");
+static_assert(part_off(1) % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0 && kTopkOff % 16 == 0,
+              "alignment");
 
 __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
   int i = 0;
@@ -79,11 +82,25 @@ __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
 #define HKV_CHECK(cond, place)
 #endif
 
+// Profiling build (-DHKV_PROFILE): thread 0 of every CTA stamps the global nanosecond timer at the
+// phase boundaries of the kernel into a buffer attached with hkv_profile_attach.
+#ifdef HKV_PROFILE
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define HKV_STAMP(k) \
+  if (P.prof && threadIdx.x == 0) P.prof[static_cast<size_t>(blockIdx.x) * kProfSlots + (k)] = global_ns();
+#else
+#define HKV_STAMP(k)
+#endif
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-template <int NT>   // 8-wide column tiles of query heads: 1 for groups up to 8, 2 for groups up to 16
-__global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(const __grid_constant__ DecodeParams P) {
+template <int NT, int W>   // NT: 8-wide column tiles of query heads (1 for groups up to 8, 2 up to 16); W: warps
+__global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __grid_constant__ DecodeParams P) {
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -91,6 +108,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
   const int csize = P.cluster;
   const bool clustered = csize > 1;
   const uint32_t crank = clustered ? cluster_ctarank() : 0u;
+  HKV_STAMP(0)
   pdl_launch_dependents();
   // "this CTA is running": has to be known before anybody touches its shared memory remotely
   if (clustered) cluster_arrive();
@@ -170,17 +188,43 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
     at_n = max(0, min(n_tiles, at_tile0 + t_per) - at_tile0);
   };
   auto sel_at = [&](int i) -> int { return sel_in_smem ? static_cast<int>(sel16[i]) : gsel[i]; };
+  // How a tile of a dynamic unit maps onto chunks: a chunk size that is a multiple of the tile holds
+  // every tile inside one chunk (one copy pair, issued by lane 0); any other size lets up to 32
+  // chunks touch a tile (one lane per chunk).  Row keys differ from (row & 7) only when the chunk
+  // size is not a multiple of 8.
+  const bool one_chunk = !contiguous && (cs % kTile) == 0;
+  const bool need_keys = !contiguous && (cs & 7) != 0;
   auto issue_attn = [&](int j) {   // whole warp; arms stage (seq0 + j) % stages with CTA tile j
     const int stage = (seq0 + j) % kDecStages;
     uint8_t* st = smem + stage * kStageBytes;
     const int v0 = (at_tile0 + j) * kTile;
     const int v1 = min(v0 + kTile, n_valid);
+    HKV_CHECK(v0 >= 0 && v0 < v1 && v1 - v0 <= kTile, 100);
+    if (contiguous || one_chunk) {
+      if (lane == 0) {
+        size_t row = static_cast<size_t>(v0);
+        if (one_chunk) {
+          const int ci = v0 / cs;
+          const int sid = sel_at(ci);
+          HKV_CHECK(sid >= 0 && sid < n_chunks, 102);
+          row = static_cast<size_t>(sid) * cs + (v0 - ci * cs);
+        }
+        HKV_CHECK(static_cast<int64_t>(row) + (v1 - v0) <= plane_rows, 103);
+#ifdef HKV_CHECKED
+        if (dead) return;
+#endif
+        const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
+        armed[stage] = seq0 + static_cast<uint32_t>(j) + 1u;
+        mbar_arrive_expect_tx(&bars[stage], 2u * bytes);
+        bulk_g2s(st, kplane + row * kRowBytes, bytes, &bars[stage]);
+        bulk_g2s(st + kTile * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
+      }
+      return;
+    }
     uint32_t* keys = reinterpret_cast<uint32_t*>(st + 2 * kTile * kRowBytes);
-    int ci = 0, p0 = 0, p1 = 0;
-    if (!contiguous) {
-      ci = v0 / cs + lane;                                 // lane-th chunk touching this tile
-      p0 = max(v0, ci * cs);
-      p1 = min(v1, (ci + 1) * cs);
+    const int ci = v0 / cs + lane;                         // lane-th chunk touching this tile
+    const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
+    if (need_keys) {
       const int v = v0 + lane;
       uint32_t key = lane & 7;
       if (v < v1) {
@@ -188,18 +232,16 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
         key = static_cast<uint32_t>(sel_at(cj) * cs + (v - cj * cs)) & 7u;
       }
       keys[lane] = key;
-    } else {
-      keys[lane] = lane & 7;
     }
-    HKV_CHECK(v0 >= 0 && v0 < v1 && v1 - v0 <= kTile, 100);
-    HKV_CHECK(contiguous ? (v1 <= plane_rows) : true, 101);
-#ifdef HKV_CHECKED
-    if (!contiguous && p0 < p1) {
+    size_t row = 0;
+    if (p0 < p1) {
       const int sid = sel_at(ci);
       HKV_CHECK(sid >= 0 && sid < n_chunks, 102);
-      HKV_CHECK(static_cast<int64_t>(sid) * cs + (p0 - ci * cs) + (p1 - p0) <= plane_rows, 103);
+      row = static_cast<size_t>(sid) * cs + (p0 - ci * cs);
+      HKV_CHECK(static_cast<int64_t>(row) + (p1 - p0) <= plane_rows, 103);
       HKV_CHECK(p0 - v0 >= 0 && p1 - v0 <= kTile, 104);
     }
+#ifdef HKV_CHECKED
     dead = __any_sync(0xffffffffu, dead);
     if (dead) return;
 #endif
@@ -209,17 +251,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       mbar_arrive_expect_tx(&bars[stage], static_cast<uint32_t>(v1 - v0) * 2u * kRowBytes);
     }
     __syncwarp();
-    if (!contiguous) {
-      if (p0 < p1) {
-        const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
-        const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
-        bulk_g2s(st + (p0 - v0) * kRowBytes, kplane + row * kRowBytes, bytes, &bars[stage]);
-        bulk_g2s(st + kTile * kRowBytes + (p0 - v0) * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
-      }
-    } else if (lane == 0) {
-      const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
-      bulk_g2s(st, kplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
-      bulk_g2s(st + kTile * kRowBytes, vplane + static_cast<size_t>(v0) * kRowBytes, bytes, &bars[stage]);
+    if (p0 < p1) {
+      const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
+      bulk_g2s(st + (p0 - v0) * kRowBytes, kplane + row * kRowBytes, bytes, &bars[stage]);
+      bulk_g2s(st + kTile * kRowBytes + (p0 - v0) * kRowBytes, vplane + row * kRowBytes, bytes, &bars[stage]);
     }
   };
 
@@ -251,14 +286,16 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
   // ---- copies that do not depend on this step's query start before the dependency wait ----
   bool attn_armed = false;
   if (scoring) {
-    for (int j = warp; j < min(sc_n, kDecStages); j += kDecWarps) issue_score(j);
+    for (int j = warp; j < min(sc_n, kDecStages); j += W) issue_score(j);
   } else if (!dynamic) {
     setup_attn(n_tok);
-    for (int j = warp; j < min(at_n, kDecStages); j += kDecWarps) issue_attn(j);
+    for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
     attn_armed = true;
   }
 
+  HKV_STAMP(1)
   pdl_wait();
+  HKV_STAMP(2)
 
   // the group's queries as B fragments of  S^T = X Q^T  (columns >= G are zero)
   uint32_t qb[8][2 * NT];
@@ -284,7 +321,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
     const uint32_t sc_addr = smem_u32(sc_smem);
     const int n_mt = sc_rows >> 4;
 
-    for (int j = warp; j < sc_n; j += kDecWarps) {
+    for (int j = warp; j < sc_n; j += W) {
       const int stage = j % kDecStages;
       const int r0 = (sc_tile0 + j) * sc_rows;
       const int nrow = min(sc_rows, n_chunks - r0);
@@ -323,9 +360,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
         v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
         v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
         const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
-        if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
-        if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
-        if (fast) {
+        if (!fast) {   // too many chunks for shared memory: the selection reads the scores from global memory
+          if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
+          if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
+        } else {
           for (int s = t; s < csize; s += 4) {
             if (c0 < n_chunks) st_cluster_f32(mapa(sc_addr + c0 * 4, s), v0);
             if (c1 < n_chunks) st_cluster_f32(mapa(sc_addr + c1 * 4, s), v1);
@@ -336,26 +374,22 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       if (j + kDecStages < sc_n) issue_score(j + kDecStages);
     }
     seq0 = static_cast<uint32_t>(sc_n);
+    HKV_STAMP(4)
 
     // every score of the unit is now on its way to every CTA of the cluster
     if (!fast) __threadfence();
     if (clustered) { cluster_arrive(); cluster_wait(); } else { __syncthreads(); }
 
-    int* hist = reinterpret_cast<int*>(smem);   // the ring is idle between the two phases
+    HKV_STAMP(5)
+    int* hist = reinterpret_cast<int*>(smem + kTopkOff);
     int* wsum = hist + 256;
     int* bc = wsum + 96;
     int emitted;
     if (identity) {
-      if (crank == 0) for (int i = tid; i < n_chunks; i += kDecWarps * 32) gsel[i] = i;
       emitted = n_chunks;
     } else if (fast) {
-      emitted = block_select_emit(
-          n_chunks, k_sel, [&](int i) { return float_key(sc_smem[i]); }, [](int) { return false; },
-          [&](int pos, int i) {
-            sel16[pos] = static_cast<uint16_t>(i);
-            if (crank == 0) gsel[pos] = i;
-          },
-          hist, wsum, bc);
+      emitted = block_topk_smem<W>(
+          sc_smem, n_chunks, k_sel, [&](int pos, int i) { sel16[pos] = static_cast<uint16_t>(i); }, hist);
       sel_in_smem = true;
     } else {
       // every CTA of the cluster writes the same list to the same place
@@ -364,15 +398,30 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
           [&](int pos, int i) { gsel[pos] = i; }, hist, wsum, bc);
     }
     __syncthreads();
-    fence_proxy_async();   // the selection's scratch in the ring is about to be overwritten by bulk copies
     int nv = emitted * cs;
     if (emitted > 0) {
       const int last = identity ? n_chunks - 1 : (sel_in_smem ? static_cast<int>(sel16[emitted - 1]) : gsel[emitted - 1]);
       if (last == n_chunks - 1) nv -= n_chunks * cs - C;   // the sequence's last chunk may be short
     }
-    if (crank == 0 && tid == 0) *n_valid_g = nv;
-    if (!do_attend) return;
+    HKV_STAMP(6)
     setup_attn(nv);
+    // the attention's first copies are what the step waits for: start them before anything else
+    if (do_attend && !dead) {
+      for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
+      attn_armed = true;
+    }
+    // what later calls may ask for (scores, selected ids, attended tokens), off the critical path
+    if (fast) {
+      const int c_per = (n_chunks + csize - 1) / csize;
+      const int c_end = min(n_chunks, static_cast<int>(crank + 1) * c_per);
+      for (int i = static_cast<int>(crank) * c_per + tid; i < c_end; i += W * 32) gscores[i] = sc_smem[i];
+    }
+    if (crank == 0) {
+      if (identity) { for (int i = tid; i < n_chunks; i += W * 32) gsel[i] = i; }
+      else if (sel_in_smem) { for (int i = tid; i < emitted; i += W * 32) gsel[i] = sel16[i]; }
+      if (tid == 0) *n_valid_g = nv;
+    }
+    if (!do_attend) return;
   } else if (dynamic) {
     setup_attn(__ldcg(n_valid_g));   // attention only: the list of an earlier selection
   }
@@ -382,9 +431,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
   // =============================================================================================
   const float sc = P.scale_log2e;
   if (!attn_armed && !dead) {
-    for (int j = warp; j < min(at_n, kDecStages); j += kDecWarps) issue_attn(j);
+    for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
   }
 
+  HKV_STAMP(7)
   float o[8][NT][4];
 #pragma unroll
   for (int dt = 0; dt < 8; ++dt) {
@@ -395,7 +445,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) { mrun[nt][0] = mrun[nt][1] = -INFINITY; lrun[nt][0] = lrun[nt][1] = 0.f; }
 
-  for (int j = warp; j < at_n && !dead; j += kDecWarps) {
+  for (int j = warp; j < at_n && !dead; j += W) {
     const int stage = (seq0 + j) % kDecStages;
     uint8_t* st = smem + stage * kStageBytes;
     const int v0 = (at_tile0 + j) * kTile;
@@ -405,14 +455,19 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       dead = true;
       break;
     }
+#ifdef HKV_PROFILE
+    if (j == 0) { HKV_STAMP(14) }
+    if (warp == 0 && j / W < 4) { HKV_STAMP(16 + 2 * (j / W)) }
+#endif
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(st + 2 * kTile * kRowBytes);
 #ifdef HKV_CHECKED
-    HKV_CHECK(keys[lane] < 8u, 110);
+    HKV_CHECK(!need_keys || keys[lane] < 8u, 110);
     HKV_CHECK(nrow >= 1, 111);
     dead = __any_sync(0xffffffffu, dead);
     if (dead) break;
 #endif
-    if (nrow < kTile) {
+    const bool partial = nrow < kTile;
+    if (partial) {
       // rows past the end were not copied: clear them so that stale bits cannot poison P*V
       for (int r = nrow; r < kTile; ++r) {
         reinterpret_cast<uint2*>(st + r * kRowBytes)[lane] = make_uint2(0u, 0u);
@@ -424,7 +479,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
     const uint32_t kbase = smem_u32(st), vbase = kbase + kTile * kRowBytes;
 
     // S^T = K Q^T : rows = tokens (two 16-row tiles), columns = query heads; the reduction over the
-    // head dimension runs as two interleaved accumulation chains
+    // head dimension runs as two interleaved accumulation chains.  Piece p of a row sits at
+    // p ^ key:  (2 kk + a_piece) ^ key = ((kk ^ (key >> 1)) << 1) | ((a_piece ^ key) & 1).
     float s[2][NT][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
@@ -435,12 +491,13 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
         s2[nt][0] = s2[nt][1] = s2[nt][2] = s2[nt][3] = 0.f;
       }
       const int r = mt * 16 + a_row;
-      const uint32_t key = keys[r];
-      const uint32_t rowaddr = kbase + r * kRowBytes;
+      const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(a_row & 7);
+      const uint32_t rowaddr = kbase + r * kRowBytes + (((a_piece ^ key) & 1u) << 4);
+      const uint32_t kx = key >> 1;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
         uint32_t a0, a1, a2, a3;
-        ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
+        ldsm_x4(a0, a1, a2, a3, rowaddr + ((kk ^ kx) << 5));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           if (kk & 1) mma_bf16(s2[nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
@@ -454,70 +511,79 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       }
     }
 
-    // online softmax per query head (this thread: heads 2t, 2t+1 of each column tile; tokens g, g+8 of each row tile)
+    // online softmax per query head (this thread: heads 2t, 2t+1 of each column tile; tokens g, g+8
+    // of each row tile); logits stay unscaled, the scale enters the exponent's fused multiply-add
     uint32_t pb[2][NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      float mx0 = -INFINITY, mx1 = -INFINITY;
+      if (partial) {
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const bool ok0 = (mt * 16 + g) < nrow, ok1 = (mt * 16 + g + 8) < nrow;
-        s[mt][nt][0] = ok0 ? s[mt][nt][0] * sc : -INFINITY;
-        s[mt][nt][1] = ok0 ? s[mt][nt][1] * sc : -INFINITY;
-        s[mt][nt][2] = ok1 ? s[mt][nt][2] * sc : -INFINITY;
-        s[mt][nt][3] = ok1 ? s[mt][nt][3] * sc : -INFINITY;
-        mx0 = fmaxf(mx0, fmaxf(s[mt][nt][0], s[mt][nt][2]));
-        mx1 = fmaxf(mx1, fmaxf(s[mt][nt][1], s[mt][nt][3]));
+        for (int mt = 0; mt < 2; ++mt) {
+          if (mt * 16 + g >= nrow) s[mt][nt][0] = s[mt][nt][1] = -INFINITY;
+          if (mt * 16 + g + 8 >= nrow) s[mt][nt][2] = s[mt][nt][3] = -INFINITY;
+        }
       }
+      float mx0 = fmaxf(fmaxf(s[0][nt][0], s[0][nt][2]), fmaxf(s[1][nt][0], s[1][nt][2]));
+      float mx1 = fmaxf(fmaxf(s[0][nt][1], s[0][nt][3]), fmaxf(s[1][nt][1], s[1][nt][3]));
 #pragma unroll
       for (int off = 4; off <= 16; off <<= 1) {
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
       }
-      const float mn0 = fmaxf(mrun[nt][0], mx0), mn1 = fmaxf(mrun[nt][1], mx1);
-      const float c0 = exp2f(mrun[nt][0] - mn0), c1 = exp2f(mrun[nt][1] - mn1);
-      mrun[nt][0] = mn0;
-      mrun[nt][1] = mn1;
+      const float mn0 = fmaxf(mrun[nt][0], mx0 * sc), mn1 = fmaxf(mrun[nt][1], mx1 * sc);
+      if (__any_sync(0xffffffffu, mn0 != mrun[nt][0] || mn1 != mrun[nt][1])) {
+        // a running maximum moved: bring the accumulators to the new reference
+        const float c0 = fast_exp2(mrun[nt][0] - mn0), c1 = fast_exp2(mrun[nt][1] - mn1);
+        mrun[nt][0] = mn0;
+        mrun[nt][1] = mn1;
+        lrun[nt][0] *= c0;
+        lrun[nt][1] *= c1;
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+          o[dt][nt][0] *= c0;
+          o[dt][nt][1] *= c1;
+          o[dt][nt][2] *= c0;
+          o[dt][nt][3] *= c1;
+        }
+      }
       float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const float p0 = exp2f(s[mt][nt][0] - mn0), p1 = exp2f(s[mt][nt][1] - mn1);
-        const float p2 = exp2f(s[mt][nt][2] - mn0), p3 = exp2f(s[mt][nt][3] - mn1);
+        const float p0 = fast_exp2(fmaf(s[mt][nt][0], sc, -mn0)), p1 = fast_exp2(fmaf(s[mt][nt][1], sc, -mn1));
+        const float p2 = fast_exp2(fmaf(s[mt][nt][2], sc, -mn0)), p3 = fast_exp2(fmaf(s[mt][nt][3], sc, -mn1));
         ps0 += p0 + p2;
         ps1 += p1 + p3;
         // P^T as the B operand of O^T += V^T P^T: tokens along k, heads along n
         pb[mt][nt][0] = movmatrix_trans(pack_bf16(p0, p1));
         pb[mt][nt][1] = movmatrix_trans(pack_bf16(p2, p3));
       }
-      lrun[nt][0] = lrun[nt][0] * c0 + ps0;
-      lrun[nt][1] = lrun[nt][1] * c1 + ps1;
-#pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
-        o[dt][nt][0] *= c0;
-        o[dt][nt][1] *= c1;
-        o[dt][nt][2] *= c0;
-        o[dt][nt][3] *= c1;
-      }
+      lrun[nt][0] += ps0;
+      lrun[nt][1] += ps1;
     }
 
     // O^T += V^T P^T : rows = head-dim (eight 16-row tiles), k = tokens (two 16-token steps)
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks) {
       const int r = ks * 16 + v_row;
-      const uint32_t key = keys[r];
-      const uint32_t rowaddr = vbase + r * kRowBytes;
+      const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(v_row & 7);
+      const uint32_t rowaddr = vbase + r * kRowBytes + (((v_piece ^ key) & 1u) << 4);
+      const uint32_t kx = key >> 1;
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         uint32_t a0, a1, a2, a3;
-        ldsm_x4_trans(a0, a1, a2, a3, rowaddr + (((2 * dt + v_piece) ^ key) << 4));
+        ldsm_x4_trans(a0, a1, a2, a3, rowaddr + ((dt ^ kx) << 5));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) mma_bf16(o[dt][nt], a0, a1, a2, a3, pb[ks][nt][0], pb[ks][nt][1]);
       }
     }
     __syncwarp();
+#ifdef HKV_PROFILE
+    if (warp == 0 && j / W < 4) { HKV_STAMP(17 + 2 * (j / W)) }
+#endif
     if (j + kDecStages < at_n) issue_attn(j + kDecStages);
   }
 
+  HKV_STAMP(8)
   // a warp that gave up tells the others, so that nobody parks results over copies still in flight
   if (__syncthreads_or(dead ? 1 : 0)) {
     // leave only after every armed stage had another bounded chance to receive its copies
@@ -529,6 +595,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
   }
   // the ring is idle from here on: it now holds the partial results
 
+  HKV_STAMP(9)
   // ---- merge the warps of this CTA ----
   // each warp parks (m, l, O): O as [16 heads][kParkStride] floats, then m[16], l[16]
   {
@@ -560,14 +627,14 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
   __syncthreads();
 
   const size_t out_row0 = static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G;
-  float* part = reinterpret_cast<float*>(smem + kPartOff);
-  float2* part_ml = reinterpret_cast<float2*>(smem + kPartOff + kMaxGroup * kHeadDim * 4);
+  float* part = reinterpret_cast<float*>(smem + (W * kParkBytes));
+  float2* part_ml = reinterpret_cast<float2*>(smem + (W * kParkBytes) + kMaxGroup * kHeadDim * 4);
   // items = (row, group of four columns): independent loads, one pass for groups up to 4, two up to 8
-  for (int item = tid; item < G * 32; item += kDecWarps * 32) {
+  for (int item = tid; item < G * 32; item += W * 32) {
     const int row = item >> 5, dq = item & 31;
-    float mw[kDecWarps], M = -INFINITY;
+    float mw[W], M = -INFINITY;
 #pragma unroll
-    for (int w2 = 0; w2 < kDecWarps; ++w2) {
+    for (int w2 = 0; w2 < W; ++w2) {
       mw[w2] = reinterpret_cast<const float*>(smem + w2 * kParkBytes)[16 * kParkStride + row];
       M = fmaxf(M, mw[w2]);
     }
@@ -575,7 +642,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
     float L = 0.f;
     if (M > -INFINITY) {
 #pragma unroll
-      for (int w2 = 0; w2 < kDecWarps; ++w2) {
+      for (int w2 = 0; w2 < W; ++w2) {
         const float* po = reinterpret_cast<const float*>(smem + w2 * kParkBytes);
         const float f = exp2f(mw[w2] - M);
         const float4 v = *reinterpret_cast<const float4*>(po + row * kParkStride + dq * 4);
@@ -600,18 +667,20 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       if (dq == 0) part_ml[row] = make_float2(M, L);
     }
   }
+  HKV_STAMP(10)
   if (!clustered) return;
 
   // ---- merge the CTAs of the cluster through distributed shared memory ----
   if (!start_waited) cluster_wait();
   cluster_arrive();
   cluster_wait();
+  HKV_STAMP(11)
   {
     const uint32_t part_addr = smem_u32(part), ml_addr = smem_u32(part_ml);
     const int total = G * kHeadDim;
     const int per = (total + csize - 1) / csize;
     const int e_end = min(total, static_cast<int>(crank + 1) * per);
-    for (int e = static_cast<int>(crank) * per + tid; e < e_end; e += kDecWarps * 32) {
+    for (int e = static_cast<int>(crank) * per + tid; e < e_end; e += W * 32) {
       const int row = e >> 7;
       float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
 #pragma unroll
@@ -643,17 +712,22 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecCtasPerSm) decode_kernel(c
       else reinterpret_cast<__nv_bfloat16*>(P.out[li])[off] = __float2bfloat16_rn(r);
     }
   }
+  HKV_STAMP(12)
   // nobody leaves while its partial may still be read
   cluster_arrive();
   cluster_wait();
+  HKV_STAMP(13)
 }
+
+// warps per CTA of each instance: the wide-group kernel needs twice the registers per thread
+constexpr int warps_of(int nt) { return nt == 1 ? kMaxWarps : 4; }
 
 template <int NT>
 void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clusters, int cluster, bool pdl,
                  cudaStream_t stream) {
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(static_cast<unsigned>(n_clusters) * cluster, 1, 1);
-  cfg.blockDim = dim3(kDecWarps * 32, 1, 1);
+  cfg.blockDim = dim3(warps_of(NT) * 32, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = stream;
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -680,16 +754,16 @@ template <int NT>
 cudaError_t configure(const ClusterCaps** out) {
   static ClusterCaps caps;
   if (!caps.ready) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<NT, warps_of(NT)>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_kernel<NT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(decode_kernel<NT, warps_of(NT)>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
     for (int c = 1; c <= kMaxCluster; c <<= 1) {
       cudaLaunchConfig_t cfg;
       cudaLaunchAttribute attr[2];
       fill_config<NT>(cfg, attr, 1, c, false, nullptr);
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<NT>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+      if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<NT, warps_of(NT)>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
       caps.max_active[c] = n;
     }
     caps.ready = true;
@@ -703,7 +777,7 @@ cudaError_t launch_nt(const DecodeParams& params, int total_units, cudaStream_t 
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
   fill_config<NT>(cfg, attr, total_units, params.cluster, params.pdl != 0, stream);
-  return cudaLaunchKernelEx(&cfg, decode_kernel<NT>, params);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<NT, warps_of(NT)>, params);
 }
 
 }  // namespace

@@ -225,4 +225,145 @@ __device__ int block_select_emit(int n, int k, KeyFn key, AlwaysFn always, EmitF
   return emitted;
 }
 
+// 2^x by the hardware approximation (relative error about 2^-22; -inf -> 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Block-wide exact top-k over finite float scores held in shared memory (the decode step's chunk
+// selection).  Selects the k largest of scores[0..n), equal scores going to the lower index, and
+// calls emit(position, index) in ascending index order; returns the number selected (= k).
+// Requires 1 <= k < n, blockDim.x = 32 * NWARPS.  scratch: kTopkScratchInts ints of shared memory.
+// Contains block barriers: every thread of the block must call it.
+//
+// One histogram pass over 256 equal-width value bins between the block's min and max score (the
+// map score -> bin is monotone, so every score in a higher bin is larger); the few scores that
+// share the bin of the k-th are then ranked exactly against each other (key, then index), which
+// yields the exact threshold element; one ordered compaction emits the result.  When that bin
+// holds more scores than the block has threads (many equal scores), the byte-wise radix
+// selection above takes over.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTopkScratchInts = 256 + 2 * 256 + 16 + 64 + 96 + 4;
+template <int NWARPS, class EmitFn>
+__device__ int block_topk_smem(const float* scores, int n, int k, EmitFn emit, int* scratch) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NTHR = NWARPS * 32;
+  int* hist = scratch;                               // [256]
+  uint32_t* cand = reinterpret_cast<uint32_t*>(scratch + 256);   // [NTHR][2]: key, index
+  int* misc = scratch + 256 + 2 * 256;               // [0] candidates gathered, [1..2] threshold key / index
+  float* red = reinterpret_cast<float*>(misc + 16);  // [NWARPS][2] min / max per warp, then [NWARPS][2] counts
+  int* wsum = misc + 16 + 64;
+  int* bc = wsum + 96;
+
+  float lo = INFINITY, hi = -INFINITY;
+  for (int i = tid; i < n; i += NTHR) { const float v = scores[i]; lo = fminf(lo, v); hi = fmaxf(hi, v); }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+  }
+  if (lane == 0) { red[2 * warp] = lo; red[2 * warp + 1] = hi; }
+  for (int i = tid; i < 256; i += NTHR) hist[i] = 0;
+  if (tid == 0) misc[0] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int w2 = 0; w2 < NWARPS; ++w2) { lo = fminf(lo, red[2 * w2]); hi = fmaxf(hi, red[2 * w2 + 1]); }
+  const float width = hi - lo;
+  const float scale = (width > 0.f && width < INFINITY) ? 255.0f / width : 0.f;
+  auto bin_of = [&](float v) { return max(0, min(255, __float2int_rd((v - lo) * scale))); };
+  for (int i = tid; i < n; i += NTHR) atomicAdd(&hist[bin_of(scores[i])], 1);
+  __syncthreads();
+
+  // every warp: the highest bin b with count(bins > b) < k <= count(bins >= b)
+  int tbin, need, cnt;
+  {
+    const int4 v0 = reinterpret_cast<const int4*>(hist)[lane * 2], v1 = reinterpret_cast<const int4*>(hist)[lane * 2 + 1];
+    const int loc[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    int tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tot += loc[j];
+    int run = tot;   // becomes the sum over lanes >= this one
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_down_sync(0xffffffffu, run, off);
+      if (lane + off < 32) run += v;
+    }
+    const int above = run - tot;
+    const bool mine = above < k && k <= above + tot;
+    int my_bin = 0, my_need = 0, my_cnt = 0;
+    if (mine) {
+      int acc = above;
+#pragma unroll
+      for (int j = 7; j >= 0; --j) {
+        if (acc < k && k <= acc + loc[j]) { my_bin = lane * 8 + j; my_need = k - acc; my_cnt = loc[j]; }
+        acc += loc[j];
+      }
+    }
+    const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+    tbin = __shfl_sync(0xffffffffu, my_bin, src);
+    need = __shfl_sync(0xffffffffu, my_need, src);
+    cnt = __shfl_sync(0xffffffffu, my_cnt, src);
+  }
+  if (cnt > NTHR) {
+    return block_select_emit(
+        n, k, [&](int i) { return float_key(scores[i]); }, [](int) { return false; }, emit, hist, wsum, bc);
+  }
+  // the scores of the threshold bin, ranked exactly: key descending, index ascending
+  for (int i = tid; i < n; i += NTHR) {
+    const float v = scores[i];
+    if (bin_of(v) == tbin) {
+      const int slot = atomicAdd(&misc[0], 1);
+      cand[2 * slot] = float_key(v);
+      cand[2 * slot + 1] = static_cast<uint32_t>(i);
+    }
+  }
+  __syncthreads();
+  if (tid < cnt) {
+    const uint32_t mk = cand[2 * tid], mi = cand[2 * tid + 1];
+    int rank = 0;
+    for (int j = 0; j < cnt; ++j) {
+      const uint32_t ok = cand[2 * j], oi = cand[2 * j + 1];
+      rank += (ok > mk) || (ok == mk && oi < mi);
+    }
+    if (rank == need - 1) { misc[1] = static_cast<int>(mk); misc[2] = static_cast<int>(mi); }
+  }
+  __syncthreads();
+  const uint32_t tkey = static_cast<uint32_t>(misc[1]);
+  const int tidx = misc[2];
+  auto taken = [&](int i) {
+    const uint32_t kv = float_key(scores[i]);
+    return kv > tkey || (kv == tkey && i <= tidx);
+  };
+  // ordered emission: warp w owns items [w * per, (w + 1) * per), per a multiple of 32
+  const int per = ((n + NWARPS - 1) / NWARPS + 31) & ~31;
+  const int beg = warp * per, end = min(n, beg + per);
+  int mine_n = 0;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    mine_n += __popc(__ballot_sync(0xffffffffu, i < end && taken(i)));
+  }
+  int* wtot = reinterpret_cast<int*>(red) + 2 * NWARPS;
+  if (lane == 0) wtot[warp] = mine_n;
+  __syncthreads();
+  int before = 0, total = 0;
+#pragma unroll
+  for (int w2 = 0; w2 < NWARPS; ++w2) {
+    const int a = wtot[w2];
+    if (w2 < warp) before += a;
+    total += a;
+  }
+  const uint32_t below = (1u << lane) - 1u;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    const bool sel = i < end && taken(i);
+    const uint32_t b = __ballot_sync(0xffffffffu, sel);
+    if (sel) emit(before + __popc(b & below), i);
+    before += __popc(b);
+  }
+  return total;
+}
+
 }  // namespace hkv

@@ -76,7 +76,11 @@ struct DecodeParams {
   void* out[kMaxMulti];
   int64_t n_valid_off[kMaxMulti];
   int64_t err_off[kMaxMulti];
+#ifdef HKV_PROFILE
+  unsigned long long* prof;   // kProfSlots time stamps (ns) per CTA, or null
+#endif
 };
+constexpr int kProfSlots = 32;
 
 // device error word helpers
 enum ErrPlace : int32_t { kErrDecodeWait = 1, kErrIndex = 2, kErrScoreWait = 3 };
