@@ -12,7 +12,8 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhkv.so")
+# HKV_LIB (development aid): path of another build of the same library, e.g. one made with HKV_NVCC_FLAGS
+_LIB_PATH = os.environ.get("HKV_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhkv.so")
 
 HKV_OK = 0
 HKV_CAUSAL_WINDOW = 1
@@ -26,7 +27,7 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
-           "hkv_topk_chunks_noalloc"]
+           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity"]
 
 
 class hkv_config(C.Structure):
@@ -76,6 +77,7 @@ def _load() -> C.CDLL:
     lib.hkv_cache_stats.argtypes = [vp, C.POINTER(hkv_stats)]
     lib.hkv_last_device_error.argtypes = [vp, i32p, i32p, vp]
     lib.hkv_topk_chunks_noalloc.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+    lib.hkv_decode_cluster_capacity.argtypes = [C.c_int32, i32p]
     lib.hkv_status_string.argtypes = [C.c_int]
     lib.hkv_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -235,6 +237,13 @@ def hkv_window_scores_offset(cache: int, b: int, h: int) -> int:
     off = C.c_size_t(0)
     _check(lib.hkv_window_scores_offset(cache, b, h, C.byref(off)), "hkv_window_scores_offset")
     return int(off.value)
+
+
+def hkv_decode_cluster_capacity(group: int) -> dict:
+    """{cluster size: clusters of the decode kernel the current device holds at once}."""
+    out = np.zeros(5, dtype=np.int32)
+    _check(lib.hkv_decode_cluster_capacity(int(group), _ptr(out, C.c_int32)), "hkv_decode_cluster_capacity")
+    return {1 << i: int(out[i]) for i in range(5)}
 
 
 def hkv_cache_stats(cache: int) -> dict:

@@ -389,6 +389,14 @@ hkv_status hkv_window_scores_offset(const hkv_cache* c, int32_t b, int32_t h, si
   return HKV_OK;
 }
 
+hkv_status hkv_decode_cluster_capacity(int32_t group, int32_t* max_active_clusters) {
+  if (!max_active_clusters || group < 1 || group > kMaxGroup) return HKV_ERR_INVALID_ARG;
+  const int* caps = nullptr;
+  if (decode_cluster_caps(group, &caps) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  for (int i = 0, c = 1; c <= kMaxCluster; c <<= 1, ++i) max_active_clusters[i] = caps[c];
+  return HKV_OK;
+}
+
 hkv_status hkv_cache_stats(const hkv_cache* c, hkv_stats* st) {
   if (!c || !st) return HKV_ERR_INVALID_ARG;
   std::memset(st, 0, sizeof(*st));

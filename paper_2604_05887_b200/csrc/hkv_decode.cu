@@ -50,7 +50,10 @@ namespace {
 constexpr int kRingBytes = kDecStages * kStageBytes;                 // staging ring
 constexpr int kParkStride = kHeadDim + 4;                            // floats per parked output row
 constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp's (O, m, l)
-constexpr int kMaxWarps = 8;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
+#ifndef HKV_DEC_WARPS
+#define HKV_DEC_WARPS 8
+#endif
+constexpr int kMaxWarps = HKV_DEC_WARPS;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
 constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
 constexpr int kSelOff = kRingBytes;                                  // uint16 ids of the selected chunks
@@ -258,6 +261,34 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
   };
 
+  // Tiles beyond the first ring-full cannot be staged yet, but their rows can already be pulled from
+  // HBM into L2, so that the later copies into the ring pay an L2 hit instead of an HBM round trip.
+  auto prefetch_attn = [&](int j) {   // whole warp; CTA tile j
+    const int v0 = (at_tile0 + j) * kTile;
+    const int v1 = min(v0 + kTile, n_valid);
+    if (contiguous || one_chunk) {
+      if (lane == 0) {
+        size_t row = static_cast<size_t>(v0);
+        if (one_chunk) {
+          const int ci = v0 / cs;
+          row = static_cast<size_t>(sel_at(ci)) * cs + (v0 - ci * cs);
+        }
+        const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
+        bulk_prefetch_l2(kplane + row * kRowBytes, bytes);
+        bulk_prefetch_l2(vplane + row * kRowBytes, bytes);
+      }
+      return;
+    }
+    const int ci = v0 / cs + lane;
+    const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
+    if (p0 < p1) {
+      const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
+      const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
+      bulk_prefetch_l2(kplane + row * kRowBytes, bytes);
+      bulk_prefetch_l2(vplane + row * kRowBytes, bytes);
+    }
+  };
+
   // ---- scoring phase: tiles of sc_rows chunk means, [sc_tile0, sc_tile0 + sc_n) for this CTA ----
   int sc_rows = 16, sc_tile0 = 0, sc_n = 0;
   if (scoring) {
@@ -290,6 +321,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   } else if (!dynamic) {
     setup_attn(n_tok);
     for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
+    for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j);
     attn_armed = true;
   }
 
@@ -408,6 +440,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     // the attention's first copies are what the step waits for: start them before anything else
     if (do_attend && !dead) {
       for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
+      for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j);
       attn_armed = true;
     }
     // what later calls may ask for (scores, selected ids, attended tokens), off the critical path
