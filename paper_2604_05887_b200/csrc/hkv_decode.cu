@@ -53,6 +53,9 @@ constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp
 #ifndef HKV_DEC_WARPS
 #define HKV_DEC_WARPS 8
 #endif
+// A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
+// latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
+constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
 constexpr int kMaxWarps = HKV_DEC_WARPS;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
 constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
@@ -321,7 +324,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   } else if (!dynamic) {
     setup_attn(n_tok);
     for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
-    for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j);
+    if (at_n <= kPrefetchMaxTiles) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
     attn_armed = true;
   }
 
@@ -440,7 +443,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     // the attention's first copies are what the step waits for: start them before anything else
     if (do_attend && !dead) {
       for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
-      for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j);
+      if (at_n <= kPrefetchMaxTiles) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
       attn_armed = true;
     }
     // what later calls may ask for (scores, selected ids, attended tokens), off the critical path
