@@ -55,6 +55,9 @@ constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp
 #endif
 // A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
 // latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
+constexpr int kRecvMlOff = 6144;   // inside the score area: (m, l) of every sender and row, after the O slices
+static_assert(kMaxCluster * 8 * 8 + kRecvMlOff <= kSelSmemChunks * 4 && 8 * kHeadDim * 4 + 4 * 4 * kMaxCluster <= kRecvMlOff,
+              "push-merge receive area fits the score area for groups up to 8");
 constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
 constexpr int kMaxWarps = HKV_DEC_WARPS;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
@@ -118,7 +121,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   pdl_launch_dependents();
   // "this CTA is running": has to be known before anybody touches its shared memory remotely
   if (clustered) cluster_arrive();
-  bool start_waited = !clustered;
+  bool bar_pending = clustered;   // an arrival on the cluster barrier that has not been waited for yet
 
   const int cid = blockIdx.x / csize;
   const int li = find_slot(P.unit_prefix, P.n, cid);
@@ -128,6 +131,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   const int G = P.group, Hq = P.n_q_heads, cs = P.chunk_size;
   const int ub = uid / P.n_kv_heads, uh = uid - ub * P.n_kv_heads;
   const bool do_select = (P.phase & kPhaseSelect) != 0, do_attend = (P.phase & kPhaseAttend) != 0;
+  constexpr bool kPushMerge = NT == 1;   // wider groups do not fit the receive area and use the pull merge
 
   // the unit's record (uniform loads, issued together)
   const int utype = up->type, C = up->C, n_tok = up->n_tok, n_chunks = up->n_chunks, k_sel = up->k_sel;
@@ -352,7 +356,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   // chunk scoring + top-k selection (dynamic units)
   // =============================================================================================
   if (scoring) {
-    if (clustered) { cluster_wait(); start_waited = true; }   // every CTA of the cluster runs: pushes are safe
+    if (clustered) { cluster_wait(); bar_pending = false; }   // every CTA of the cluster runs: pushes are safe
     const uint32_t sc_addr = smem_u32(sc_smem);
     const int n_mt = sc_rows >> 4;
 
@@ -458,6 +462,8 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       if (tid == 0) *n_valid_g = nv;
     }
     if (!do_attend) return;
+    // "my selection is done": from here on my score area is free to receive the peers' partial results
+    if (clustered && kPushMerge) { cluster_arrive_relaxed(); bar_pending = true; }
   } else if (dynamic) {
     setup_attn(__ldcg(n_valid_g));   // attention only: the list of an earlier selection
   }
@@ -665,6 +671,14 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   const size_t out_row0 = static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G;
   float* part = reinterpret_cast<float*>(smem + (W * kParkBytes));
   float2* part_ml = reinterpret_cast<float2*>(smem + (W * kParkBytes) + kMaxGroup * kHeadDim * 4);
+  // Push merge (groups up to 8): the output's G*128 elements are dealt to the cluster's CTAs in
+  // slices of `per`; every CTA sends each owner its share of (m, l, O) into the owner's score area,
+  // which is idle by now (peers have signalled the end of their selection), so that after one
+  // cluster barrier each owner reduces from its own shared memory and nobody has to wait again.
+  const int total = G * kHeadDim;
+  const int per = (((total + csize - 1) / csize) + 3) & ~3;
+  const uint32_t recv_acc = smem_u32(smem + kScoresOff), recv_ml = recv_acc + kRecvMlOff;
+  if (clustered && kPushMerge && bar_pending) { cluster_wait(); bar_pending = false; }
   // items = (row, group of four columns): independent loads, one pass for groups up to 4, two up to 8
   for (int item = tid; item < G * 32; item += W * 32) {
     const int row = item >> 5, dq = item & 31;
@@ -698,6 +712,13 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
         pk.y = pack_bf16(acc.z * inv, acc.w * inv);
         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(P.out[li]) + off) = pk;
       }
+    } else if (kPushMerge) {
+      const int e0 = row * kHeadDim + dq * 4;
+      const int owner = e0 / per;
+      st_cluster_f32x4(mapa(recv_acc + (static_cast<int>(crank) * per + (e0 - owner * per)) * 4, owner), acc);
+      if (dq == 0) {
+        for (int s2 = 0; s2 < csize; ++s2) st_cluster_f32x2(mapa(recv_ml + (static_cast<int>(crank) * G + row) * 8, s2), M, L);
+      }
     } else {
       *reinterpret_cast<float4*>(part + row * kHeadDim + dq * 4) = acc;
       if (dq == 0) part_ml[row] = make_float2(M, L);
@@ -706,8 +727,50 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   HKV_STAMP(10)
   if (!clustered) return;
 
+  if (kPushMerge) {
+    cluster_arrive();
+    cluster_wait();
+    HKV_STAMP(11)
+    const float* racc = reinterpret_cast<const float*>(smem + kScoresOff);
+    const float2* rml = reinterpret_cast<const float2*>(smem + kScoresOff + kRecvMlOff);
+    const int e_lo = static_cast<int>(crank) * per, e_hi = min(total, e_lo + per);
+    for (int e = e_lo + tid; e < e_hi; e += W * 32) {
+      const int row = e >> 7, le = e - e_lo;
+      float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+        if (s2 < csize) {
+          const float2 ml = rml[s2 * G + row];
+          ms[s2] = ml.x;
+          ls[s2] = ml.y;
+          av[s2] = racc[s2 * per + le];
+        } else {
+          ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f;
+        }
+      }
+      float M = -INFINITY;
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) M = fmaxf(M, ms[s2]);
+      float acc = 0.f, L = 0.f;
+      if (M > -INFINITY) {
+#pragma unroll
+        for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+          const float f = exp2f(ms[s2] - M);
+          acc += av[s2] * f;
+          L += ls[s2] * f;
+        }
+      }
+      const float r = L > 0.f ? acc / L : 0.f;
+      const size_t off = out_row0 * kHeadDim + e;
+      if (P.out_f32) reinterpret_cast<float*>(P.out[li])[off] = r;
+      else reinterpret_cast<__nv_bfloat16*>(P.out[li])[off] = __float2bfloat16_rn(r);
+    }
+    HKV_STAMP(13)
+    return;   // nothing of this CTA is read remotely after the barrier above
+  }
+
   // ---- merge the CTAs of the cluster through distributed shared memory ----
-  if (!start_waited) cluster_wait();
+  if (bar_pending) cluster_wait();
   cluster_arrive();
   cluster_wait();
   HKV_STAMP(11)
