@@ -16,17 +16,25 @@
 //     takes up to 64 staged means and computes  S^T = M Q^T  (rows = chunks, columns = the group's
 //     query heads) on tensor cores; the chunk score is the float32 sum over the group's heads.
 //     Scores are pushed into the shared memory of every CTA of the cluster (distributed shared
-//     memory), a cluster barrier follows, and each CTA then runs the same exact radix selection on
-//     its own copy, so that every CTA knows the ascending list of selected chunks without a
-//     round trip through global memory.
+//     memory), a cluster barrier follows, and each CTA then runs the same exact selection on its
+//     own copy (a 256-bin value histogram finds the bin of the k-th score, the few scores of that
+//     bin are ranked exactly by key and index), so that every CTA knows the ascending list of
+//     selected chunks without a round trip through global memory.  The lists later calls may ask
+//     for (scores, ids, token count) are written to global memory only after the attention's first
+//     copies have been issued.
 //   every unit, attention:  the unit's token list (static: the compacted rows; dynamic: the rows of
 //     the selected chunks) is cut into 32-token tiles, dealt to the cluster's CTAs as contiguous
 //     ranges.  Per tile:  S^T = K Q^T  (rows = tokens, columns = query heads, so the group shares
 //     every loaded KV tile and no tensor-core row is padding), online softmax in float32 (base-2
-//     exponent), P^T moved into operand layout with movmatrix,  O^T += V^T P^T.
-//   merge:  the warps of a CTA are combined in shared memory; the CTAs of the cluster read each
-//     other's partial (m, l, O) through distributed shared memory, each producing a slice of the
-//     output — fixed order, no atomics, deterministic.
+//     exponent, accumulators rescaled only when a running maximum moves), P^T moved into operand
+//     layout with movmatrix,  O^T += V^T P^T.  A CTA with a short list asks L2 for its tiles beyond
+//     the first ring-full as soon as it knows them.
+//   merge:  the warps of a CTA are combined in shared memory.  Groups up to 8: every CTA then sends
+//     each owner CTA its share of (m, l, O) into the owner's idle score area (distributed shared
+//     memory stores), one cluster barrier follows, and each owner reduces its slice of the output
+//     from its own shared memory in CTA-rank order.  Wider groups: the CTAs read each other's
+//     partials after the barrier and a second barrier keeps them alive.  Fixed order, no atomics:
+//     deterministic.
 //
 // Programmatic dependent launch.  Nothing the kernel does before griddepcontrol.wait depends on the
 // step's query or on an earlier decode launch: it reads the unit table, arms the barriers and has
