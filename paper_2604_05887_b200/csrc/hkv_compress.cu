@@ -173,23 +173,31 @@ __global__ void __launch_bounds__(kWsWarps * 32)
   }
 }
 
-__global__ void window_rowreduce_kernel(const char* cache, const float2* stats, float2* final_stats, int n_tiles_max,
-                                        int Rpad) {
+// Combines the per-tile (max, sum) of every window row into the row's final (max, sum): one warp per
+// row, lanes stride the column tiles.
+constexpr int kRowReduceWarps = 8;
+__global__ void __launch_bounds__(kRowReduceWarps * 32)
+    window_rowreduce_kernel(const char* cache, const float2* stats, float2* final_stats, int n_tiles_max, int Rpad) {
   const Header* hdr = reinterpret_cast<const Header*>(cache);
-  const Unit* u = unit_of(cache, hdr, false, blockIdx.x, nullptr);
+  const Unit* u = unit_of(cache, hdr, false, blockIdx.y, nullptr);
   const int R = hdr->obs_window * hdr->group;
   const int n_tiles = (u->C + kWsTile - 1) / kWsTile;
-  for (int r = threadIdx.x; r < R; r += blockDim.x) {
-    const float2* st = stats + static_cast<size_t>(blockIdx.x) * n_tiles_max * Rpad + r;
-    float M = -INFINITY;
-    for (int jt = 0; jt < n_tiles; ++jt) M = fmaxf(M, st[static_cast<size_t>(jt) * Rpad].x);
-    float Z = 0.f;
-    for (int jt = 0; jt < n_tiles; ++jt) {
-      const float2 v = st[static_cast<size_t>(jt) * Rpad];
-      if (v.x > -INFINITY) Z += v.y * exp2f(v.x - M);
-    }
-    final_stats[static_cast<size_t>(blockIdx.x) * Rpad + r] = make_float2(M, Z);
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * kRowReduceWarps + (threadIdx.x >> 5);
+  if (r >= R) return;
+  const float2* st = stats + static_cast<size_t>(blockIdx.y) * n_tiles_max * Rpad + r;
+  float M = -INFINITY;
+  for (int jt = lane; jt < n_tiles; jt += 32) M = fmaxf(M, st[static_cast<size_t>(jt) * Rpad].x);
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+  float Z = 0.f;
+  for (int jt = lane; jt < n_tiles; jt += 32) {
+    const float2 v = st[static_cast<size_t>(jt) * Rpad];
+    if (v.x > -INFINITY) Z += v.y * exp2f(v.x - M);
   }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
+  if (lane == 0) final_stats[static_cast<size_t>(blockIdx.y) * Rpad + r] = make_float2(M, Z);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -286,25 +294,45 @@ __global__ void __launch_bounds__(256)
   }
 }
 
-// Chunk means: thread = one channel; float32 running sum over the chunk's tokens in order, float32
-// division by the chunk's own length, round-to-nearest-even to bf16.
-__global__ void __launch_bounds__(kHeadDim) chunk_means_kernel(char* cache, const __nv_bfloat16* kin) {
+// Chunk means: half a warp per chunk, lane = eight channels (one 16-byte piece of a key row); every
+// channel keeps its own float32 running sum over the chunk's tokens IN ORDER, then a float32 division
+// by the chunk's own length and round-to-nearest-even to bf16 — the arithmetic the method's metadata
+// is defined with, so the result is bit-exact whatever the launch shape.  Rows of consecutive tokens
+// are independent loads, so four are kept in flight.
+constexpr int kMeanWarps = 8;
+__global__ void __launch_bounds__(kMeanWarps * 32) chunk_means_kernel(char* cache, const uint4* kin) {
   const Header* hdr = reinterpret_cast<const Header*>(cache);
   const Unit* u = unit_of(cache, hdr, true, blockIdx.y, nullptr);
-  const int cs = hdr->chunk_size, C = u->C, d = threadIdx.x;
-  const __nv_bfloat16* kp =
-      kin + (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * static_cast<size_t>(hdr->max_seq_len) * kHeadDim;
-  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(cache + u->summ_off);
-  for (int cc = 0; cc < 8; ++cc) {
-    const int c = blockIdx.x * 8 + cc;
-    if (c >= u->n_chunks) break;
-    const int t0 = c * cs, t1 = min(t0 + cs, C);
-    float acc = 0.f;
-    for (int tk = t0; tk < t1; ++tk) acc = __fadd_rn(acc, __bfloat162float(kp[static_cast<size_t>(tk) * kHeadDim + d]));
-    // 16-byte piece p of chunk c is stored at position p ^ (c & 7), like K/V rows
-    out[static_cast<size_t>(c) * kHeadDim + ((((d >> 3) ^ (c & 7)) << 3) | (d & 7))] =
-        __float2bfloat16_rn(__fdiv_rn(acc, static_cast<float>(t1 - t0)));
+  const int cs = hdr->chunk_size, C = u->C;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, sub = lane & 15;
+  const int c = (blockIdx.x * kMeanWarps + warp) * 2 + (lane >> 4);
+  if (c >= u->n_chunks) return;
+  const uint4* kp = kin + (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * static_cast<size_t>(hdr->max_seq_len) * 16;
+  const int t0 = c * cs, t1 = min(t0 + cs, C);
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  auto add_row = [&](const uint4& r) {
+    acc[0] = __fadd_rn(acc[0], bf16_lo(r.x)); acc[1] = __fadd_rn(acc[1], bf16_hi(r.x));
+    acc[2] = __fadd_rn(acc[2], bf16_lo(r.y)); acc[3] = __fadd_rn(acc[3], bf16_hi(r.y));
+    acc[4] = __fadd_rn(acc[4], bf16_lo(r.z)); acc[5] = __fadd_rn(acc[5], bf16_hi(r.z));
+    acc[6] = __fadd_rn(acc[6], bf16_lo(r.w)); acc[7] = __fadd_rn(acc[7], bf16_hi(r.w));
+  };
+  int tk = t0;
+  for (; tk + 4 <= t1; tk += 4) {
+    const uint4 r0 = kp[static_cast<size_t>(tk) * 16 + sub], r1 = kp[static_cast<size_t>(tk + 1) * 16 + sub];
+    const uint4 r2 = kp[static_cast<size_t>(tk + 2) * 16 + sub], r3 = kp[static_cast<size_t>(tk + 3) * 16 + sub];
+    add_row(r0); add_row(r1); add_row(r2); add_row(r3);
   }
+  for (; tk < t1; ++tk) add_row(kp[static_cast<size_t>(tk) * 16 + sub]);
+  const float len = static_cast<float>(t1 - t0);
+  uint4 o;
+  o.x = pack_bf16(__fdiv_rn(acc[0], len), __fdiv_rn(acc[1], len));
+  o.y = pack_bf16(__fdiv_rn(acc[2], len), __fdiv_rn(acc[3], len));
+  o.z = pack_bf16(__fdiv_rn(acc[4], len), __fdiv_rn(acc[5], len));
+  o.w = pack_bf16(__fdiv_rn(acc[6], len), __fdiv_rn(acc[7], len));
+  // 16-byte piece p of chunk c is stored at position p ^ (c & 7), like K/V rows
+  reinterpret_cast<uint4*>(cache + u->summ_off)[static_cast<size_t>(c) * 16 + (sub ^ (c & 7))] = o;
 }
 
 }  // namespace
@@ -321,7 +349,8 @@ cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, co
   window_scores_kernel<0><<<grid, kWsWarps * 32, 0, stream>>>(
       cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
       n_col_tiles_max, Rpad);
-  window_rowreduce_kernel<<<hdr.n_static, 256, 0, stream>>>(cache, stats, fin, n_col_tiles_max, Rpad);
+  window_rowreduce_kernel<<<dim3((R + kRowReduceWarps - 1) / kRowReduceWarps, hdr.n_static), kRowReduceWarps * 32, 0, stream>>>(
+      cache, stats, fin, n_col_tiles_max, Rpad);
   window_scores_kernel<1><<<grid, kWsWarps * 32, 0, stream>>>(
       cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
       n_col_tiles_max, Rpad);
@@ -348,8 +377,8 @@ cudaError_t launch_build_dynamic(char* cache, const void* k, const void* v, cons
   if (hdr.n_dynamic == 0) return cudaSuccess;
   dim3 grid((max_rows + 63) / 64, hdr.n_dynamic);
   gather_rows_kernel<<<grid, 256, 0, stream>>>(cache, static_cast<const uint4*>(k), static_cast<const uint4*>(v), 1);
-  dim3 grid2((max_chunks + 7) / 8, hdr.n_dynamic);
-  chunk_means_kernel<<<grid2, kHeadDim, 0, stream>>>(cache, static_cast<const __nv_bfloat16*>(k));
+  dim3 grid2((max_chunks + kMeanWarps * 2 - 1) / (kMeanWarps * 2), hdr.n_dynamic);
+  chunk_means_kernel<<<grid2, kMeanWarps * 32, 0, stream>>>(cache, static_cast<const uint4*>(k));
   return cudaGetLastError();
 }
 
