@@ -158,6 +158,27 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
 
 hkv_status hkv_cache_destroy(hkv_cache* cache);
 
+/* Top-down budget allocation (Section 3.2, both paragraphs): from a total token budget to the
+ * per-head budgets hkv_plan / hkv_compress take.  Host arithmetic in double precision, no device.
+ *   n_heads      heads the total is shared by (all layers' KV heads of one sequence, in any fixed order)
+ *   head_type    host u8 [n_heads]   0 = static, 1 = dynamic (Section 3.1)
+ *   scores       host f64 [n_heads]  text-centric sparsity score S_{l,h} >= 0 of each head (only static
+ *                                    heads' entries are read); NULL = all equal
+ *   total_budget B_total in tokens, >= n_heads
+ *   r            share coefficient of the dynamic heads, 0 < r <= B_total / (B_bar * N_dyna)
+ *   alpha        in [0, 1]: weight of the uniform base budget against the score-proportional one
+ *   flags        HKV_BUDGET_PAD_POW2: round the dynamic per-head budget up to a power of two
+ *   budgets_out  host int32 [n_heads]
+ * Head-type level:  B_bar = B_total / (N_stat + N_dyna);  B_dyna = ceil(r * B_bar * N_dyna);
+ * B_stat = B_total - B_dyna.  Static head:  b = ceil(alpha * B_stat / N_stat + (1 - alpha) * B_stat * S~),
+ * S~ = S / sum of S over all static heads.  Dynamic head:  ceil(B_dyna / N_dyna), the same for all.
+ * Errors: HKV_ERR_BUDGET if r breaks its bound, if the total cannot give every head one token, or
+ * alpha is outside [0, 1]. */
+#define HKV_BUDGET_PAD_POW2 1u
+hkv_status hkv_allocate_budgets(int32_t n_heads, const uint8_t* head_type, const double* scores,
+                                int64_t total_budget, double r, double alpha, uint32_t flags,
+                                int32_t* budgets_out);
+
 /* Chunk scoring + top-k for one dynamic head WITHOUT any caller- or library-allocated scratch.
  * (The paper has no counterpart: this is a packaging variant of the selection step of
  * hkv_select_chunks.)  It exists for callers that cannot allocate device memory where they call

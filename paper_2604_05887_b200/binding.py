@@ -27,7 +27,7 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
-           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity"]
+           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets"]
 
 
 class hkv_config(C.Structure):
@@ -78,6 +78,8 @@ def _load() -> C.CDLL:
     lib.hkv_last_device_error.argtypes = [vp, i32p, i32p, vp]
     lib.hkv_topk_chunks_noalloc.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
     lib.hkv_decode_cluster_capacity.argtypes = [C.c_int32, i32p]
+    lib.hkv_allocate_budgets.argtypes = [C.c_int32, u8p, C.POINTER(C.c_double), C.c_int64, C.c_double, C.c_double,
+                                         C.c_uint32, i32p]
     lib.hkv_status_string.argtypes = [C.c_int]
     lib.hkv_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -244,6 +246,22 @@ def hkv_decode_cluster_capacity(group: int) -> dict:
     out = np.zeros(5, dtype=np.int32)
     _check(lib.hkv_decode_cluster_capacity(int(group), _ptr(out, C.c_int32)), "hkv_decode_cluster_capacity")
     return {1 << i: int(out[i]) for i in range(5)}
+
+
+HKV_BUDGET_PAD_POW2 = 1
+
+
+def hkv_allocate_budgets(head_type, scores, total_budget: int, r: float, alpha: float, flags: int = 0) -> np.ndarray:
+    """Per-head token budgets from a total budget (host arithmetic; see hkv.h)."""
+    ht = _u8(head_type).ravel()
+    out = np.zeros(ht.size, dtype=np.int32)
+    sp = None
+    if scores is not None:
+        sc = np.ascontiguousarray(np.asarray(scores, dtype=np.float64).ravel())
+        sp = _ptr(sc, C.c_double)
+    _check(lib.hkv_allocate_budgets(ht.size, _ptr(ht, C.c_uint8), sp, int(total_budget), float(r), float(alpha),
+                                    int(flags), _ptr(out, C.c_int32)), "hkv_allocate_budgets")
+    return out
 
 
 def hkv_cache_stats(cache: int) -> dict:
