@@ -65,6 +65,7 @@ typedef struct {
   int32_t obs_window;    /* w: length of the observation window (Appendix A)                   */
   float softmax_scale;   /* 0 -> 1/sqrt(head_dim); used by S_w and by decode attention         */
   uint32_t flags;
+  int32_t append_capacity; /* tokens hkv_append may add to every sequence after compression (0 = none) */
 } hkv_config;
 
 typedef struct hkv_cache hkv_cache; /* opaque; host metadata of one layer's compressed cache */
@@ -155,6 +156,22 @@ hkv_status hkv_attend(hkv_cache* cache, const void* q, void* out, void* stream);
  *   q_dev, out_dev    caller-owned device staging buffers of the same sizes */
 hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_host, void* q_dev,
                                 void* out_dev, void* stream);
+
+/* Adds the token just generated to the compressed cache of one layer (Appendix A: the GPU KV buffer
+ * is "updated" as decoding proceeds; Section 3.3: the buffer is "updated by dynamic heads during
+ * decoding").  Reading taken here, the paper giving no rule: the new token's key / value row of
+ *   a static head   is appended to its condensed cache and is always retained (it is the most
+ *                   recent context);
+ *   a dynamic head  joins the chunked sequence: it goes to the open last chunk (or opens a new one),
+ *                   whose metadata is recomputed as the float32 running sum of its keys in token
+ *                   order / its length, rounded to bf16 — bit-identical to building the metadata
+ *                   of the longer sequence from scratch; the number of chunks loaded per step
+ *                   follows the unchanged budget.
+ *   k_new, v_new  dev bf16 [B, Hkv, d]   the new token's key and value of every KV head
+ * Every sequence grows by one token per call, at most hkv_config.append_capacity times
+ * (HKV_ERR_WORKSPACE afterwards).  Enqueued on `stream`, no synchronisation; must not overlap a
+ * decode call on the same cache. */
+hkv_status hkv_append(hkv_cache* cache, const void* k_new, const void* v_new, void* stream);
 
 hkv_status hkv_cache_destroy(hkv_cache* cache);
 

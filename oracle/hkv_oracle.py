@@ -236,6 +236,30 @@ def compress_layer(L, token_scores: Optional[np.ndarray] = None, scale: Optional
     return cache
 
 
+def append_token(L, cache: OracleCache, k_new: np.ndarray, v_new: np.ndarray) -> None:
+    """Adds the token just generated (k_new, v_new: uint16 [B, Hkv, d]) to one layer's compressed cache
+    (Appendix A / Section 3.3 only say the GPU buffer is "updated"; reading taken: a static head always
+    retains the new token, a dynamic head's chunking simply covers the longer sequence, its metadata being
+    what chunk_summaries gives for that longer sequence, and the number of chunks per step follows the
+    unchanged budget).  L.k / L.v must have room (max_seq_len > seq_len); L and cache are updated in place."""
+    for b in range(L.batch):
+        C = int(L.seq_lens[b])
+        assert C < L.k.shape[2], "no room for another token"
+        L.k[b, :, C] = k_new[b]
+        L.v[b, :, C] = v_new[b]
+        L.seq_lens[b] = C + 1
+        for h in range(L.n_kv_heads):
+            hd = cache.heads.get((b, h))
+            if hd is None:
+                continue
+            hd.C = C + 1
+            if hd.kind == 0:
+                hd.keep = np.concatenate([hd.keep, np.array([C], dtype=np.int64)])
+            else:
+                hd.summaries = chunk_summaries(L.k[b, h, :C + 1], L.chunk_size)
+                hd.n_sel = n_selected_chunks(int(L.budgets[b, h]), L.chunk_size, hd.summaries.shape[0])
+
+
 def decode_layer(L, cache: OracleCache, q: np.ndarray, scale: Optional[float] = None,
                  chunk_override: Optional[Dict[Tuple[int, int], np.ndarray]] = None,
                  keep_override: Optional[Dict[Tuple[int, int], np.ndarray]] = None):

@@ -27,13 +27,14 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
-           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets"]
+           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append"]
 
 
 class hkv_config(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("max_seq_len", C.c_int32), ("chunk_size", C.c_int32),
-                ("obs_window", C.c_int32), ("softmax_scale", C.c_float), ("flags", C.c_uint32)]
+                ("obs_window", C.c_int32), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
+                ("append_capacity", C.c_int32)]
 
 
 class hkv_stats(C.Structure):
@@ -69,6 +70,7 @@ def _load() -> C.CDLL:
     lib.hkv_attend.argtypes = [vp, vp, vp, vp]
     lib.hkv_decode_attn_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hkv_cache_destroy.argtypes = [vp]
+    lib.hkv_append.argtypes = [vp, vp, vp, vp]
     for name in ("hkv_get_static_indices", "hkv_get_selected_chunks"):
         getattr(lib, name).argtypes = [vp, C.c_int32, C.c_int32, i32p, C.c_int32, i32p, vp]
     lib.hkv_get_chunk_scores.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(C.c_float), C.c_int32, i32p, vp]
@@ -131,9 +133,9 @@ def _stream(stream) -> Optional[int]:
 
 
 def make_config(batch, n_q_heads, n_kv_heads, head_dim, max_seq_len, chunk_size, obs_window,
-                softmax_scale: float = 0.0, flags: int = 0) -> hkv_config:
+                softmax_scale: float = 0.0, flags: int = 0, append_capacity: int = 0) -> hkv_config:
     return hkv_config(batch, n_q_heads, n_kv_heads, head_dim, max_seq_len, chunk_size, obs_window,
-                      softmax_scale, flags)
+                      softmax_scale, flags, append_capacity)
 
 
 def hkv_plan(cfg: hkv_config, seq_lens, head_type, budgets):
@@ -194,6 +196,11 @@ def hkv_topk_chunks_noalloc(q, means, k: int, out_ids, stream=None) -> None:
     q: bf16 CUDA [group, 128]; means: bf16 CUDA [n_chunks, 128] plain row-major; out_ids: int32 CUDA [min(k, n_chunks)]."""
     _check(lib.hkv_topk_chunks_noalloc(_dev(q), _dev(means), int(q.shape[0]), int(means.shape[0]), int(k),
                                        _dev(out_ids), _stream(stream)), "hkv_topk_chunks_noalloc")
+
+
+def hkv_append(cache: int, k_new, v_new, stream=None) -> None:
+    """k_new, v_new: bf16 CUDA [B, Hkv, d], the new token's key / value of every KV head."""
+    _check(lib.hkv_append(cache, _dev(k_new), _dev(v_new), _stream(stream)), "hkv_append")
 
 
 def hkv_cache_destroy(cache: int) -> None:

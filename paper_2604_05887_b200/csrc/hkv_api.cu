@@ -26,6 +26,7 @@ hkv_status check_config(const hkv_config* cfg) {
   if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32)) return HKV_ERR_INVALID_ARG;
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return HKV_ERR_INVALID_ARG;
   if (static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads > 60000) return HKV_ERR_UNSUPPORTED;
+  if (cfg->append_capacity < 0 || cfg->append_capacity > (1 << 24)) return HKV_ERR_SHAPE;
   return HKV_OK;
 }
 
@@ -63,9 +64,12 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
       u.type = head_type[b * Hkv + h];
       u.b = b; u.h = h; u.C = seq_lens[b];
       u.budget = std::min(budgets[b * Hkv + h], u.C);
+      u.budget_raw = budgets[b * Hkv + h];
+      const int cap = cfg->append_capacity;
       if (u.type == 0) {
         u.n_tok = u.budget;
-        u.plane_rows = u.n_tok;
+        u.plane_rows = u.n_tok + cap;
+        u.cap_sel = u.n_tok + cap;
         c.max_static_rows = std::max(c.max_static_rows, u.plane_rows);
         max_C = std::max(max_C, u.C);
         H.n_static++;
@@ -74,12 +78,14 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
         u.n_chunks = (u.C + cs - 1) / cs;
         u.k_sel = std::min(u.n_chunks, (u.budget + cs - 1) / cs);
         const int64_t nt = static_cast<int64_t>(u.k_sel) * cs;
-        const int64_t pr = static_cast<int64_t>(u.n_chunks) * cs;
+        u.cap_chunks = static_cast<int32_t>((static_cast<int64_t>(u.C) + cap + cs - 1) / cs);
+        u.cap_sel = static_cast<int32_t>(std::min<int64_t>(u.cap_chunks, (static_cast<int64_t>(std::min<int64_t>(u.budget_raw, static_cast<int64_t>(u.C) + cap)) + cs - 1) / cs));
+        const int64_t pr = static_cast<int64_t>(u.cap_chunks) * cs;
         if (pr > 0x7FFFFFF0ll) return HKV_ERR_UNSUPPORTED;
         u.n_tok = static_cast<int32_t>(nt);
         u.plane_rows = static_cast<int32_t>(pr);
         c.max_dyn_rows = std::max(c.max_dyn_rows, u.plane_rows);
-        c.max_chunks = std::max(c.max_chunks, u.n_chunks);
+        c.max_chunks = std::max(c.max_chunks, u.cap_chunks);
         H.n_dynamic++;
         c.algo_bytes += 2ll * kRowBytes * std::min<int64_t>(nt, u.C) + static_cast<int64_t>(kRowBytes) * u.n_chunks;
         c.summary_bytes += static_cast<int64_t>(kRowBytes) * u.n_chunks;
@@ -102,10 +108,11 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
   H.err_off = off;       off = align_up(off + 8);
   for (auto& u : c.units) {
     u.idx_off = off;
-    off = align_up(off + 4ll * std::max(1, u.type == 0 ? u.n_tok : u.k_sel));
+    off = align_up(off + 4ll * std::max(1, u.cap_sel));
     if (u.type == 1) {
-      u.scores_off = off;  off = align_up(off + 4ll * u.n_chunks);
-      u.summ_off = off;    off = align_up(off + static_cast<int64_t>(kRowBytes) * u.n_chunks);
+      u.scores_off = off;    off = align_up(off + 4ll * u.cap_chunks);
+      u.summ_off = off;      off = align_up(off + static_cast<int64_t>(kRowBytes) * u.cap_chunks);
+      u.tail_sum_off = off;  off = align_up(off + 4ll * kHeadDim);
     }
   }
   for (auto& u : c.units) {
@@ -177,6 +184,7 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
     if (st != HKV_OK) { delete c; return st; }
     c->dev_base = static_cast<char*>(cache_mem);
     c->fresh = true;
+    c->appended = 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const Header& H = c->hdr;
 
@@ -323,6 +331,37 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
   hkv_status st = hkv_decode_attn(cache, q_dev, out_dev, stream);
   if (st != HKV_OK) return st;
   if (cudaMemcpyAsync(out_host, out_dev, n * out_elt, cudaMemcpyDeviceToHost, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  return HKV_OK;
+}
+
+hkv_status hkv_append(hkv_cache* c, const void* k_new, const void* v_new, void* stream) {
+  if (!c || !k_new || !v_new) return HKV_ERR_INVALID_ARG;
+  if (c->appended >= c->cfg.append_capacity) return HKV_ERR_WORKSPACE;
+  if (launch_append(c->dev_base, k_new, v_new, c->hdr, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return HKV_ERR_CUDA;
+  }
+  // the host mirror follows the same rule as the kernel, so that no call has to wait for the device
+  const int cs = c->cfg.chunk_size;
+  c->retained = c->algo_bytes = c->summary_bytes = 0;
+  c->max_tiles = 1;
+  for (auto& u : c->units) {
+    u.C += 1;
+    if (u.type == 0) {
+      u.n_tok += 1;
+      c->algo_bytes += 2ll * kRowBytes * u.n_tok;
+    } else {
+      u.n_chunks = (u.C + cs - 1) / cs;
+      u.k_sel = std::min(u.n_chunks, (std::min(u.budget_raw, u.C) + cs - 1) / cs);
+      u.n_tok = u.k_sel * cs;
+      c->algo_bytes += 2ll * kRowBytes * std::min(u.n_tok, u.C) + static_cast<int64_t>(kRowBytes) * u.n_chunks;
+      c->summary_bytes += static_cast<int64_t>(kRowBytes) * u.n_chunks;
+    }
+    c->retained += std::min(u.n_tok, u.C);
+    c->max_tiles = std::max(c->max_tiles, (u.n_tok + kTile - 1) / kTile);
+  }
+  c->appended += 1;
+  c->fresh = true;   // the next decode launch must not start before this kernel has finished
   return HKV_OK;
 }
 

@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(256)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = lane & 15;
   const bool is_v = lane >= 16;
-  const int rows = u->plane_rows;
+  const int rows = dynamic ? u->plane_rows : u->n_tok;   // (rows kept for appended tokens are written by the append kernel)
   const int32_t* idx = reinterpret_cast<const int32_t*>(cache + u->idx_off);
   const size_t plane_in = (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * static_cast<size_t>(hdr->max_seq_len);
   uint4* dst_plane = reinterpret_cast<uint4*>(cache + (is_v ? u->v_off : u->k_off));
@@ -333,6 +333,63 @@ __global__ void __launch_bounds__(kMeanWarps * 32) chunk_means_kernel(char* cach
   o.w = pack_bf16(__fdiv_rn(acc[6], len), __fdiv_rn(acc[7], len));
   // 16-byte piece p of chunk c is stored at position p ^ (c & 7), like K/V rows
   reinterpret_cast<uint4*>(cache + u->summ_off)[static_cast<size_t>(c) * 16 + (sub ^ (c & 7))] = o;
+  if (c == u->n_chunks - 1) {
+    // running sum of the open last chunk, continued by appended tokens (a full chunk leaves nothing open)
+    float* tail = reinterpret_cast<float*>(cache + u->tail_sum_off) + sub * 8;
+    const bool open = (t1 - t0) < cs;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tail[j] = open ? acc[j] : 0.f;
+  }
+}
+
+// Adds one token to every unit: the key / value rows go to the end of the unit's planes (static: the
+// condensed cache, position recorded in the kept list; dynamic: row C of the chunk-major store), a
+// dynamic unit's open chunk gets its running sum and mean updated (or a new chunk is opened), and the
+// unit's record is advanced.  One CTA of 128 threads per unit; thread = channel.
+__global__ void __launch_bounds__(kHeadDim)
+    append_kernel(char* cache, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new) {
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  Unit* u = reinterpret_cast<Unit*>(cache + kUnitsOff) + blockIdx.x;
+  const int d = threadIdx.x, cs = hdr->chunk_size;
+  const int C = u->C;
+  const bool dynamic = u->type != 0;
+  const int row = dynamic ? C : u->n_tok;
+  if (row >= u->plane_rows) {   // no room left (the host refuses this before launching)
+    if (d == 0) {
+      int32_t* err = reinterpret_cast<int32_t*>(cache + hdr->err_off);
+      if (atomicCAS(&err[0], 0, HKV_ERR_INDEX) == 0) err[1] = kErrIndex;
+    }
+    return;
+  }
+  const size_t in = (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * kHeadDim + d;
+  const __nv_bfloat16 kv = k_new[in], vv = v_new[in];
+  const size_t out = static_cast<size_t>(row) * kHeadDim + ((((d >> 3) ^ (row & 7)) << 3) | (d & 7));
+  reinterpret_cast<__nv_bfloat16*>(cache + u->k_off)[out] = kv;
+  reinterpret_cast<__nv_bfloat16*>(cache + u->v_off)[out] = vv;
+  int n_chunks = u->n_chunks;
+  if (dynamic) {
+    const int c = C / cs;                       // chunk the new token falls into
+    const int len = C - c * cs + 1;
+    float* tail = reinterpret_cast<float*>(cache + u->tail_sum_off);
+    const float sum = __fadd_rn(len == 1 ? 0.f : tail[d], __bfloat162float(kv));
+    tail[d] = (len == cs) ? 0.f : sum;          // a chunk that just filled up leaves nothing open
+    reinterpret_cast<__nv_bfloat16*>(cache + u->summ_off)[static_cast<size_t>(c) * kHeadDim + ((((d >> 3) ^ (c & 7)) << 3) | (d & 7))] =
+        __float2bfloat16_rn(__fdiv_rn(sum, static_cast<float>(len)));
+    n_chunks = c + 1;
+  }
+  __syncthreads();   // every thread has read the record
+  if (d == 0) {
+    u->C = C + 1;
+    if (dynamic) {
+      u->n_chunks = n_chunks;
+      const int k_sel = min(n_chunks, (min(u->budget_raw, C + 1) + cs - 1) / cs);
+      u->k_sel = k_sel;
+      u->n_tok = k_sel * cs;
+    } else {
+      reinterpret_cast<int32_t*>(cache + u->idx_off)[u->n_tok] = C;   // position of the new token
+      u->n_tok = u->n_tok + 1;
+    }
+  }
 }
 
 }  // namespace
@@ -379,6 +436,12 @@ cudaError_t launch_build_dynamic(char* cache, const void* k, const void* v, cons
   gather_rows_kernel<<<grid, 256, 0, stream>>>(cache, static_cast<const uint4*>(k), static_cast<const uint4*>(v), 1);
   dim3 grid2((max_chunks + kMeanWarps * 2 - 1) / (kMeanWarps * 2), hdr.n_dynamic);
   chunk_means_kernel<<<grid2, kMeanWarps * 32, 0, stream>>>(cache, static_cast<const uint4*>(k));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(char* cache, const void* k_new, const void* v_new, const Header& hdr, cudaStream_t stream) {
+  append_kernel<<<hdr.n_units, kHeadDim, 0, stream>>>(cache, static_cast<const __nv_bfloat16*>(k_new),
+                                                      static_cast<const __nv_bfloat16*>(v_new));
   return cudaGetLastError();
 }
 

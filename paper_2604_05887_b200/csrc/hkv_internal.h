@@ -33,15 +33,18 @@ struct Unit {
   int32_t n_tok;       // static: kept tokens; dynamic: k_sel * cs (upper bound of attended tokens)
   int32_t n_chunks;    // dynamic: ceil(C / cs)
   int32_t k_sel;       // dynamic: chunks loaded per step
-  int32_t plane_rows;  // rows of the K (and V) plane held in the cache
-  int32_t pad0[3];
+  int32_t plane_rows;  // rows of the K (and V) plane held in the cache (capacity, including room for appended tokens)
+  int32_t budget_raw;  // the caller's budget before clamping to the sequence length
+  int32_t cap_chunks;  // dynamic: chunk means / scores the cache has room for
+  int32_t cap_sel;     // entries the index list has room for
   int64_t k_off, v_off;    // byte offsets (from the cache base) of the K / V planes
   int64_t summ_off;        // dynamic: bf16 chunk means [n_chunks, d], 16-byte pieces permuted like K/V rows
   int64_t idx_off;         // static: int32 kept positions [n_tok]; dynamic: int32 chunk ids [k_sel]
   int64_t scores_off;      // dynamic: float32 chunk scores [n_chunks] (decode scratch)
   int64_t ws_scores_off;   // static: float32 s_w [C] inside the compress workspace
+  int64_t tail_sum_off;    // dynamic: float32 [d] running key sum of the open last chunk (zero when it is full)
 };
-static_assert(sizeof(Unit) == 96, "Unit layout");
+static_assert(sizeof(Unit) == 104, "Unit layout");
 
 // Device-side table of contents, at offset 0 of cache_mem.  Unit[n_units] follows at kUnitsOff.
 struct Header {
@@ -105,6 +108,7 @@ cudaError_t launch_gather_static(char* cache, const void* k, const void* v, cons
                                  int max_rows, cudaStream_t stream);
 cudaError_t launch_build_dynamic(char* cache, const void* k, const void* v, const Header& hdr,
                                  int max_rows, int max_chunks, cudaStream_t stream);
+cudaError_t launch_append(char* cache, const void* k_new, const void* v_new, const Header& hdr, cudaStream_t stream);
 size_t decode_smem_bytes();
 
 }  // namespace hkv
@@ -117,5 +121,6 @@ struct hkv_cache {
   size_t cache_bytes, workspace_bytes;
   int64_t kv_bytes, summary_bytes, algo_bytes, retained;
   int max_static_rows, max_dyn_rows, max_chunks, max_tiles;
-  bool fresh;   // no decode launch has followed the compression yet
+  bool fresh;   // no decode launch has followed the last compression / append yet
+  int appended; // tokens added by hkv_append so far
 };

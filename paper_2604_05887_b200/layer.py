@@ -23,9 +23,9 @@ class LayerCache:
     L: any object with the fields of hkv_inputs.LayerInputs (host numpy arrays)."""
 
     def __init__(self, L, flags: int = 0, token_scores: np.ndarray | None = None, softmax_scale: float = 0.0,
-                 device="cuda", keep_workspace: bool = False, k_dev=None, v_dev=None):
+                 device="cuda", keep_workspace: bool = False, k_dev=None, v_dev=None, append_capacity: int = 0):
         self.cfg = hkv.make_config(L.batch, L.n_q_heads, L.n_kv_heads, L.head_dim, L.max_seq_len, L.chunk_size,
-                                   L.obs_window, softmax_scale, flags)
+                                   L.obs_window, softmax_scale, flags, append_capacity)
         self.flags = flags
         self.shape = (L.batch, L.n_q_heads, L.head_dim)
         self.device = device
@@ -55,6 +55,11 @@ class LayerCache:
             out = self.new_out()
         hkv.hkv_decode_attn(self.handle, q, out)
         return out
+
+    def append(self, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+        """Adds the new token's key / value ([B, Hkv, d] bf16 CUDA tensors) to the cache."""
+        hkv.hkv_append(self.handle, k_new, v_new)
+        self.stats = hkv.hkv_cache_stats(self.handle)
 
     def window_scores(self, b: int, h: int, C: int) -> np.ndarray:
         """float32 s_w the compression computed (needs keep_workspace=True)."""
