@@ -230,3 +230,30 @@ def test_cfg4_full_size_cell_sampled(P):
     L = hi.cfg4(0.10, 0.5, 32)
     rep = P.compare_layer(L, units=[(0, 0), (5, 1), (9, 2), (15, 3)])
     print("cfg4 cell", rep)
+
+
+@pytest.mark.parametrize("budget,sf,cs,units", [
+    (1.00, 0.5, 64, [(0, 0), (7, 2), (15, 3)]),       # full budget: both head types equal full-cache attention
+    (0.05, 0.25, 16, [(1, 1), (8, 0), (14, 2)]),      # 2048 chunk means per head, k = 103
+    (0.50, 0.75, 128, [(2, 3), (9, 1), (13, 0)]),
+])
+def test_cfg4_full_size_more_cells_sampled(P, budget, sf, cs, units):
+    """More cells of the B=16, 32768-token sweep at full size, in the launch shape the sweep times."""
+    L = hi.cfg4(budget, sf, cs)
+    rep = P.compare_layer(L, units=units)
+    if budget >= 1.0:
+        # the oracle's answer at 100 % is itself pinned to textbook attention (test_oracle_pins); check one unit here too
+        b, h = units[0]
+        C, G = int(L.seq_lens[b]), L.group
+        f = lambda u: torch.from_numpy(np.ascontiguousarray(u)).view(torch.bfloat16).to(torch.float64)
+        from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+        lc = LayerCache(L, flags=2)
+        out = lc.decode(to_device_bf16(L.q[0])).cpu().numpy()
+        Q = f(L.q[0][b, h * G:(h + 1) * G])[None, :, None, :]
+        K = f(L.k[b, h, :C])[None, None].expand(1, G, C, 128)
+        V = f(L.v[b, h, :C])[None, None].expand(1, G, C, 128)
+        ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V)[0, :, 0].numpy()
+        P.check_outputs(out[b, h * G:(h + 1) * G], ref, "full budget vs textbook attention")
+        lc.close()
+    print("cfg4 cell", budget, sf, cs, {k: rep[k] for k in ("max_abs", "mean_abs", "swaps_dynamic")})
+
