@@ -361,7 +361,7 @@ def main():
     kv_in_bytes = 0
     for layer in range(n_layers):
         t0 = time.perf_counter()
-        L = layer_inputs(args.workload, layer, args.seed + 1000 * rank, threads)
+        L = layer_inputs(args.workload, layer, args.seed + 1000 * rank, threads)   # = replicas.replica_seed(seed, rank)
         t_gen += time.perf_counter() - t0
         k_dev, v_dev = to_device_bf16(L.k, dev), to_device_bf16(L.v, dev)
         torch.cuda.synchronize()
@@ -417,10 +417,11 @@ def main():
             step_e2e()
         stream.synchronize()
 
+        from paper_2604_05887_b200 import replicas
+
         def barrier():
             torch.cuda.synchronize()
-            if dist is not None:
-                dist.barrier()
+            replicas.barrier()
             torch.cuda.synchronize()
 
         def timed(g, n):
@@ -431,11 +432,7 @@ def main():
                 g.replay()
             b.record(stream)
             barrier()
-            ms = a.elapsed_time(b)
-            if dist is not None:
-                t = torch.tensor([ms], device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms = float(t.item())
+            ms, _, _ = replicas.aggregate_step(a.elapsed_time(b), algo_bytes, dev)   # the slowest rank's time
             return ms
 
         for _ in range(max(args.warmup, 3)):

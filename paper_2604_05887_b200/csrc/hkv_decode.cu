@@ -61,11 +61,11 @@ constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp
 #ifndef HKV_DEC_WARPS
 #define HKV_DEC_WARPS 8
 #endif
-// A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
-// latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
 constexpr int kRecvMlOff = 6144;   // inside the score area: (m, l) of every sender and row, after the O slices
 static_assert(kMaxCluster * 8 * 8 + kRecvMlOff <= kSelSmemChunks * 4 && 8 * kHeadDim * 4 + 4 * 4 * kMaxCluster <= kRecvMlOff,
               "push-merge receive area fits the score area for groups up to 8");
+// A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
+// latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
 constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
 constexpr int kMaxWarps = HKV_DEC_WARPS;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
