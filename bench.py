@@ -405,10 +405,10 @@ def main():
         out_all = torch.empty_like(out_host, device=dev)
 
         def step_e2e():
-            q_all.copy_(q_host, non_blocking=True)
-            for i, lc in enumerate(caches):
-                hkv.hkv_decode_attn(lc.handle, q_all[i], out_all[i])
-            out_host.copy_(out_all, non_blocking=True)
+            # the library's host-buffer entry point for a whole step: all layers' queries (pinned host) ->
+            # device in one transfer, one decode launch per layer, all outputs -> pinned host, every copy
+            # enqueued by the C-ABI call itself
+            hkv.hkv_decode_step_host([lc.handle for lc in caches], q_host, out_host, q_all, out_all)
 
         step_e2e()
         stream.synchronize()
@@ -505,7 +505,7 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
         "e2e": {"value": world_bytes / t_e2e / 1e9, "unit": "GB/s", "us_per_step": t_e2e * 1e6,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "how": "pinned host queries -> device, 28 x hkv_decode_attn, outputs -> pinned host, all inside the timed graph"},
+                "how": "hkv_decode_step_host: pinned host queries of all layers -> device, one decode launch per layer, outputs -> pinned host, copies enqueued by the C-ABI call, all inside the timed graph (the per-layer host entry point hkv_decode_attn_host costs two PCIe round trips per layer: 990 us/step)"},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk.summary(),
         "device_error": [code, detail],

@@ -173,6 +173,16 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
  * decode call on the same cache. */
 hkv_status hkv_append(hkv_cache* cache, const void* k_new, const void* v_new, void* stream);
 
+/* One decode step of a whole model with HOST buffers (Appendix A's per-step procedure, layer after
+ * layer): the queries of all n layers are copied to the device in one transfer, one hkv_decode_attn
+ * launch per layer follows (caches[i] with layer i's slice, in order), and all outputs return in
+ * one transfer — everything enqueued on `stream`.
+ *   q_host, out_host  host [n, B, Hq, d] (pinned for truly asynchronous copies); bf16 / float32 as for hkv_decode_attn
+ *   q_dev, out_dev    caller-owned device staging buffers of the same sizes
+ * All caches must share one geometry (batch, heads, output type). */
+hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void* q_host, void* out_host,
+                                void* q_dev, void* out_dev, void* stream);
+
 hkv_status hkv_cache_destroy(hkv_cache* cache);
 
 /* Top-down budget allocation (Section 3.2, both paragraphs): from a total token budget to the

@@ -27,7 +27,7 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
-           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append"]
+           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append", "hkv_decode_step_host"]
 
 
 class hkv_config(C.Structure):
@@ -70,6 +70,7 @@ def _load() -> C.CDLL:
     lib.hkv_attend.argtypes = [vp, vp, vp, vp]
     lib.hkv_decode_attn_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hkv_cache_destroy.argtypes = [vp]
+    lib.hkv_decode_step_host.argtypes = [C.POINTER(vp), C.c_int32, vp, vp, vp, vp, vp]
     lib.hkv_append.argtypes = [vp, vp, vp, vp]
     for name in ("hkv_get_static_indices", "hkv_get_selected_chunks"):
         getattr(lib, name).argtypes = [vp, C.c_int32, C.c_int32, i32p, C.c_int32, i32p, vp]
@@ -186,6 +187,15 @@ def hkv_decode_attn_host(cache: int, q_host, out_host, q_dev, out_dev, stream=No
         raise ValueError("q_host and out_host must be contiguous CPU tensors")
     _check(lib.hkv_decode_attn_host(cache, q_host.data_ptr(), out_host.data_ptr(), _dev(q_dev), _dev(out_dev),
                                     _stream(stream)), "hkv_decode_attn_host")
+
+
+def hkv_decode_step_host(caches: Sequence[int], q_host, out_host, q_dev, out_dev, stream=None) -> None:
+    """One decode step over all layers with host buffers [n, B, Hq, d] (see hkv.h)."""
+    n = len(caches)
+    if q_host.is_cuda or out_host.is_cuda or not q_host.is_contiguous() or not out_host.is_contiguous():
+        raise ValueError("q_host and out_host must be contiguous CPU tensors")
+    _check(lib.hkv_decode_step_host((C.c_void_p * n)(*caches), n, q_host.data_ptr(), out_host.data_ptr(), _dev(q_dev),
+                                    _dev(out_dev), _stream(stream)), "hkv_decode_step_host")
 
 
 HKV_NOALLOC_MAX_CHUNKS = 65536

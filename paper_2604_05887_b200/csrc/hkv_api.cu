@@ -334,6 +334,29 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
   return HKV_OK;
 }
 
+hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void* q_host, void* out_host, void* q_dev,
+                                void* out_dev, void* stream) {
+  if (!caches || n < 1 || !q_host || !out_host || !q_dev || !out_dev) return HKV_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!caches[i]) return HKV_ERR_INVALID_ARG;
+    const hkv_config &a = caches[i]->cfg, &b = caches[0]->cfg;
+    if (a.batch != b.batch || a.n_q_heads != b.n_q_heads || a.head_dim != b.head_dim ||
+        ((a.flags ^ b.flags) & HKV_OUT_F32))
+      return HKV_ERR_SHAPE;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t per = static_cast<size_t>(caches[0]->cfg.batch) * caches[0]->cfg.n_q_heads * caches[0]->cfg.head_dim;
+  const size_t out_elt = (caches[0]->hdr.flags & HKV_OUT_F32) ? 4 : 2;
+  if (cudaMemcpyAsync(q_dev, q_host, per * 2 * n, cudaMemcpyHostToDevice, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  for (int i = 0; i < n; ++i) {
+    hkv_status st = hkv_decode_attn(caches[i], static_cast<const char*>(q_dev) + per * 2 * i,
+                                    static_cast<char*>(out_dev) + per * out_elt * i, stream);
+    if (st != HKV_OK) return st;
+  }
+  if (cudaMemcpyAsync(out_host, out_dev, per * out_elt * n, cudaMemcpyDeviceToHost, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  return HKV_OK;
+}
+
 hkv_status hkv_append(hkv_cache* c, const void* k_new, const void* v_new, void* stream) {
   if (!c || !k_new || !v_new) return HKV_ERR_INVALID_ARG;
   if (c->appended >= c->cfg.append_capacity) return HKV_ERR_WORKSPACE;

@@ -257,3 +257,27 @@ def test_cfg4_full_size_more_cells_sampled(P, budget, sf, cs, units):
         lc.close()
     print("cfg4 cell", budget, sf, cs, {k: rep[k] for k in ("max_abs", "mean_abs", "swaps_dynamic")})
 
+
+def test_host_buffer_entry_points_equal_device_calls():
+    """hkv_decode_attn_host (one layer) and hkv_decode_step_host (all layers, one transfer each way)."""
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    Ls = [hi.cfg1(layer=l, C=2048, block=256, n_steps=1) for l in range(3)]
+    lcs = [LayerCache(L) for L in Ls]
+    qs = [to_device_bf16(L.q[0]) for L in Ls]
+    ref = [lc.decode(q).clone() for lc, q in zip(lcs, qs)]
+    torch.cuda.synchronize()
+    q_host = torch.stack([q.cpu() for q in qs]).pin_memory()
+    out_host = torch.zeros_like(q_host).pin_memory()
+    q_dev, out_dev = torch.empty_like(q_host, device="cuda"), torch.empty_like(q_host, device="cuda")
+    hkv.hkv_decode_step_host([lc.handle for lc in lcs], q_host, out_host, q_dev, out_dev)
+    torch.cuda.synchronize()
+    for i in range(3):
+        assert torch.equal(out_host[i].view(torch.int16), ref[i].cpu().view(torch.int16))
+    one = torch.zeros_like(q_host[1]).pin_memory()
+    hkv.hkv_decode_attn_host(lcs[1].handle, q_host[1], one, q_dev[1], out_dev[1])
+    torch.cuda.synchronize()
+    assert torch.equal(one.view(torch.int16), ref[1].cpu().view(torch.int16))
+    for lc in lcs:
+        lc.close()
+
