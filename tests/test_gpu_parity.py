@@ -281,3 +281,22 @@ def test_host_buffer_entry_points_equal_device_calls():
     for lc in lcs:
         lc.close()
 
+
+def test_more_units_than_clusters_fit(P):
+    """200 (sequence, head) units: the launch falls back to one CTA per unit (no cluster, no cross-CTA merge)."""
+    L = small(B=50, C=260, cs=16, w=8, budget=0.3, n_steps=1)
+    rep = P.compare_layer(L)
+    assert rep["stats"]["n_splits"] == 200
+
+
+def test_unit_counts_that_select_every_cluster_size(P):
+    """1, 2, 4, 8 and 16 CTAs per unit (the launch picks the largest size that fits all units in one wave)."""
+    from paper_2604_05887_b200 import binding as hkv
+    caps = hkv.hkv_decode_cluster_capacity(7)
+    seen = set()
+    for B in (1, 3, 6, 12, 30, 50):
+        L = small(B=B, C=1500, cs=32, w=8, budget=0.5, n_steps=1, ragged=False)
+        rep = P.compare_layer(L, units=[(0, 0), (B - 1, 3), (B // 2, 1), (B // 2, 2)])
+        seen.add(rep["stats"]["n_splits"] // (4 * B))
+    assert seen >= {1, 2, 4, 8}, (seen, caps)
+
