@@ -79,8 +79,9 @@ typedef struct {
   int64_t cache_bytes;           /* bytes of cache_mem in use                                  */
   int64_t workspace_bytes;       /* bytes of compress workspace required                       */
   int32_t n_static, n_dynamic;   /* (b, h) units of each type                                  */
-  int32_t n_splits;              /* CTAs of the flash-decode launch                            */
-  int32_t launches_per_decode;   /* kernels one hkv_decode_attn enqueues                       */
+  int32_t n_splits;              /* CTAs of a decode launch on this cache alone (units x cluster size) */
+  int32_t launches_per_decode;   /* kernels one hkv_decode_attn enqueues (1: score, select, attend and
+                                    merge are one kernel)                                      */
 } hkv_stats;
 
 /* Sizes of the two caller-owned device buffers, from HOST inputs only (no device work, no sync).
@@ -130,8 +131,11 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
  * Dynamic head: score_c = sum over the group's query heads of <q_g, mean_c> (float32), top-k with
  * ties to the lower chunk id, softmax attention over the tokens of the selected chunks.  Static
  * head: softmax attention over its kept tokens.  Heads are independent.  Allocates nothing, never
- * synchronises, results are deterministic.  Calls on the same cache must not overlap on the GPU
- * (they share the cache's scratch). */
+ * synchronises, results are deterministic.  q must be 4-byte and out 16-byte aligned.  Calls on the
+ * same cache must not overlap on the GPU (they share the cache's scratch).  One kernel launch; when
+ * it follows another decode launch on the stream it is launched with programmatic stream
+ * serialisation: it may start early, but reads q and writes anything only once everything enqueued
+ * before it has completed. */
 hkv_status hkv_decode_attn(hkv_cache* cache, const void* q, void* out, void* stream);
 
 /* Decode several layers' caches with ONE launch sequence: queries q[i] / outputs out[i] belong to
