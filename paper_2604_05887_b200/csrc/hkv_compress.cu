@@ -206,12 +206,11 @@ __global__ void __launch_bounds__(kRowReduceWarps * 32)
 // does not exceed the window, the last `budget` tokens.  One CTA per static unit, ascending output.
 // ---------------------------------------------------------------------------------------------
 constexpr int kKeepThreads = 1024;
+constexpr int kKeepScratchInts = keyed_scratch_ints(kKeepThreads);
 
 __global__ void __launch_bounds__(kKeepThreads)
     static_select_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text) {
-  __shared__ int hist[256];
-  __shared__ int wsum[96];
-  __shared__ int bc[4];
+  __shared__ __align__(16) int scratch[kKeepScratchInts];
   __shared__ int s_ntext;
 
   const Header* hdr = reinterpret_cast<const Header*>(cache);
@@ -238,22 +237,21 @@ __global__ void __launch_bounds__(kKeepThreads)
   int emitted;
   if (budget <= w) {
     const int start = C - budget;
-    emitted = block_select_emit(
-        C, 0, [](int) { return 0u; }, [&](int i) { return i >= start; }, [&](int pos, int i) { out[pos] = i; }, hist, wsum,
-        bc);
+    emitted = block_topk_keyed<kKeepThreads>(
+        C, 0, [](int) { return 0u; }, [&](int i) { return i >= start; }, [&](int pos, int i) { out[pos] = i; }, scratch);
   } else {
     const int room = budget - w;
     const bool rank_text = n_text >= room;       // window + text do not fit: rank the text tokens
     const int k = rank_text ? room : room - n_text;
-    emitted = block_select_emit(
+    emitted = block_topk_keyed<kKeepThreads>(
         C, k,
         [&](int i) {
           if (i >= hist_end) return 0u;
           const bool is_t = txt[i] != 0;
           return (is_t == rank_text) ? float_key(scores[i]) : 0u;
         },
-        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, [&](int pos, int i) { out[pos] = i; }, hist,
-        wsum, bc);
+        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, [&](int pos, int i) { out[pos] = i; },
+        scratch);
   }
   if (tid == 0) {
     reinterpret_cast<int32_t*>(cache + hdr->n_valid_off)[uid] = emitted;

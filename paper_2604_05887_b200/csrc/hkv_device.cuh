@@ -383,4 +383,142 @@ __device__ int block_topk_smem(const float* scores, int n, int k, EmitFn emit, i
   return total;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Block-wide exact selection over keyed items that need not sit in shared memory (the static
+// heads' Top-M visual tokens: tens of thousands of candidates with a heavy-tailed score).  Same
+// contract as block_select_emit: items with always(i) are emitted, and of the items with
+// key(i) != 0 the k with the largest keys, equal keys going to the lower index; emission in
+// ascending index order; returns the number emitted.  Requires k <= number of candidates.
+//
+// One 1024-bin histogram over (key - min key) >> shift (order-preserving keys of floats are close to
+// log-spaced, which suits a heavy tail), exact ranking of the threshold bin's items by (key, index),
+// one ordered compaction.  Falls back to the byte-wise radix selection when the threshold bin
+// holds more items than the block has threads or when k = 0.
+// scratch: kKeyedScratchInts(NTHR) ints of shared memory.
+// ---------------------------------------------------------------------------------------------
+constexpr int kKeyedBins = 1024;
+constexpr int keyed_scratch_ints(int nthr) { return kKeyedBins + 2 * nthr + 8 + 64 + 256 + 96 + 4; }
+template <int NTHR, class KeyFn, class AlwaysFn, class EmitFn>
+__device__ int block_topk_keyed(int n, int k, KeyFn key, AlwaysFn always, EmitFn emit, int* scratch) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NWARPS = NTHR / 32;
+  int* hist = scratch;                                                   // [1024]
+  uint32_t* cand = reinterpret_cast<uint32_t*>(scratch + kKeyedBins);   // [NTHR][2]
+  int* misc = scratch + kKeyedBins + 2 * NTHR;                           // [0] candidates, [1..2] threshold, [4] min, [5] max
+  int* wtot = misc + 8;                                                  // [NWARPS]
+  int* fb_hist = wtot + 64;                                              // fallback's scratch
+  int* fb_wsum = fb_hist + 256;
+  int* fb_bc = fb_wsum + 96;
+  if (k <= 0) return block_select_emit(n, k, key, always, emit, fb_hist, fb_wsum, fb_bc);
+
+  for (int i = tid; i < kKeyedBins; i += NTHR) hist[i] = 0;
+  if (tid == 0) { misc[0] = 0; misc[4] = -1; misc[5] = 0; }   // min as unsigned: 0xFFFFFFFF
+  __syncthreads();
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+  for (int i = tid; i < n; i += NTHR) {
+    const uint32_t kv = key(i);
+    if (kv != 0u) { kmin = min(kmin, kv); kmax = max(kmax, kv); }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) {
+    atomicMin(reinterpret_cast<unsigned int*>(&misc[4]), kmin);
+    atomicMax(reinterpret_cast<unsigned int*>(&misc[5]), kmax);
+  }
+  __syncthreads();
+  kmin = static_cast<uint32_t>(misc[4]);
+  kmax = static_cast<uint32_t>(misc[5]);
+  const uint32_t range = kmax - kmin;
+  const int shift = max(0, 32 - __clz(range | 1u) - 10);      // (range >> shift) < 1024
+  auto bin_of = [&](uint32_t kv) { return static_cast<int>((kv - kmin) >> shift); };
+  for (int i = tid; i < n; i += NTHR) {
+    const uint32_t kv = key(i);
+    if (kv != 0u) atomicAdd(&hist[bin_of(kv)], 1);
+  }
+  __syncthreads();
+  // every warp: the highest bin b with count(bins > b) < k <= count(bins >= b); lane owns 32 bins
+  int tbin, need, cnt;
+  {
+    int loc[32], tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int4 v = reinterpret_cast<const int4*>(hist)[lane * 8 + j];
+      loc[4 * j] = v.x; loc[4 * j + 1] = v.y; loc[4 * j + 2] = v.z; loc[4 * j + 3] = v.w;
+      tot += v.x + v.y + v.z + v.w;
+    }
+    int run = tot;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_down_sync(0xffffffffu, run, off);
+      if (lane + off < 32) run += v;
+    }
+    const int above = run - tot;
+    const bool mine = above < k && k <= above + tot;
+    int my_bin = 0, my_need = 0, my_cnt = 0;
+    if (mine) {
+      int acc = above;
+#pragma unroll
+      for (int j = 31; j >= 0; --j) {
+        if (acc < k && k <= acc + loc[j]) { my_bin = lane * 32 + j; my_need = k - acc; my_cnt = loc[j]; }
+        acc += loc[j];
+      }
+    }
+    const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+    tbin = __shfl_sync(0xffffffffu, my_bin, src);
+    need = __shfl_sync(0xffffffffu, my_need, src);
+    cnt = __shfl_sync(0xffffffffu, my_cnt, src);
+  }
+  if (cnt > NTHR) return block_select_emit(n, k, key, always, emit, fb_hist, fb_wsum, fb_bc);
+  for (int i = tid; i < n; i += NTHR) {
+    const uint32_t kv = key(i);
+    if (kv != 0u && bin_of(kv) == tbin) {
+      const int slot = atomicAdd(&misc[0], 1);
+      cand[2 * slot] = kv;
+      cand[2 * slot + 1] = static_cast<uint32_t>(i);
+    }
+  }
+  __syncthreads();
+  if (tid < cnt) {
+    const uint32_t mk = cand[2 * tid], mi = cand[2 * tid + 1];
+    int rank = 0;
+    for (int j = 0; j < cnt; ++j) {
+      const uint32_t ok = cand[2 * j], oi = cand[2 * j + 1];
+      rank += (ok > mk) || (ok == mk && oi < mi);
+    }
+    if (rank == need - 1) { misc[1] = static_cast<int>(mk); misc[2] = static_cast<int>(mi); }
+  }
+  __syncthreads();
+  const uint32_t tkey = static_cast<uint32_t>(misc[1]);
+  const int tidx = misc[2];
+  auto taken = [&](int i) {
+    if (always(i)) return true;
+    const uint32_t kv = key(i);
+    return kv != 0u && (kv > tkey || (kv == tkey && i <= tidx));
+  };
+  const int per = ((n + NWARPS - 1) / NWARPS + 31) & ~31;
+  const int beg = warp * per, end = min(n, beg + per);
+  int mine_n = 0;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    mine_n += __popc(__ballot_sync(0xffffffffu, i < end && taken(i)));
+  }
+  if (lane == 0) wtot[warp] = mine_n;
+  __syncthreads();
+  int before = 0, total = 0;
+  for (int w2 = 0; w2 < NWARPS; ++w2) {
+    const int a = wtot[w2];
+    if (w2 < warp) before += a;
+    total += a;
+  }
+  const uint32_t below = (1u << lane) - 1u;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    const bool sel = i < end && taken(i);
+    const uint32_t b = __ballot_sync(0xffffffffu, sel);
+    if (sel) emit(before + __popc(b & below), i);
+    before += __popc(b);
+  }
+  return total;
+}
+
 }  // namespace hkv
