@@ -300,3 +300,23 @@ def test_unit_counts_that_select_every_cluster_size(P):
         seen.add(rep["stats"]["n_splits"] // (4 * B))
     assert seen >= {1, 2, 4, 8}, (seen, caps)
 
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes(P, case):
+    """Seeded random geometry: batch, lengths, chunk size, window, group size, per-head budgets and types."""
+    rng = np.random.default_rng(1000 + case)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 7, 8, 12, 16]))
+    B = int(rng.integers(1, 7))
+    C = int(rng.integers(80, 3000))
+    cs = int(rng.choice([1, 3, 8, 16, 20, 32, 64, 96, 128, 500]))
+    w = int(rng.integers(1, min(48, C - 5 * B - 1)))
+    L = hi.tiny(seed=2000 + case, B=B, C=C, chunk_size=cs, w=w, Hq=G * Hkv, Hkv=Hkv, d=128, budget_fraction=0.2,
+                n_steps=2, ragged=bool(case & 1))
+    L.head_type = rng.integers(0, 2, size=(B, Hkv)).astype(np.uint8)
+    L.budgets = rng.integers(1, C + 50, size=(B, Hkv)).astype(np.int32)
+    units = [(b, h) for b in range(B) for h in range(Hkv)]
+    if len(units) > 8:
+        units = [units[i] for i in rng.choice(len(units), size=8, replace=False)]
+    P.compare_layer(L, units=units)
+
