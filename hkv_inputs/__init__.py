@@ -41,7 +41,7 @@ HEAD_DIM = 128
 OBS_WINDOW = 32
 
 # tensor ids for the Philox key
-_T_K, _T_V, _T_QOBS, _T_Q, _T_MISC, _T_MEAN, _T_DIR = range(7)
+_T_K, _T_V, _T_QOBS, _T_Q, _T_MISC, _T_MEAN, _T_DIR, _T_QTEXT = range(8)
 
 
 # --------------------------------------------------------------------------------------------
@@ -335,3 +335,25 @@ def tiny(seed: int = 11, B: int = 2, C: int = 96, chunk_size: int = 8, w: int = 
                 _normal_bits(_rng(seed, 0, _T_V, b, h), (Cb, d)))
     return _make_layer("tiny", seed, 0, B, C, seq_lens, is_text, chunk_size, 0.5, budget_fraction,
                        n_steps, kv, Hq=Hq, Hkv=Hkv, d=d, w=w, threads=1, head_type=head_type)
+
+
+def text_queries(L: LayerInputs, n_text: int, seed: int = 5, gain: float = 1.5, n_anchor: int = 4,
+                 ragged: bool = True):
+    """Queries of the prompt's text tokens for head classification: (q_text uint16 [B, n_text, Hq, d],
+    counts int32 [B]).  Every kv head gets a focus level in [0, 1] (cycling 0, 1/3, 2/3, 1 over b * Hkv + h):
+    its text queries are N(0,1) noise plus focus * gain * one of `n_anchor` anchor keys of that head, so
+    that the heads' attention rows range from diffuse to sharply peaked."""
+    B, Hq, Hkv, d, G = L.batch, L.n_q_heads, L.n_kv_heads, L.head_dim, L.group
+    counts = np.array([max(1, n_text - (3 * b if ragged else 0)) for b in range(B)], dtype=np.int32)
+    q = np.zeros((B, n_text, Hq, d), dtype=np.float32)
+    for b in range(B):
+        C = int(L.seq_lens[b])
+        for h in range(Hkv):
+            rng = _rng(seed, L.layer, _T_QTEXT, b, h)
+            focus = ((b * Hkv + h) % 4) / 3.0
+            anchors = rng.choice(C, size=min(n_anchor, C), replace=False)
+            x = rng.standard_normal((n_text, G, d), dtype=np.float32)
+            pick = anchors[rng.integers(0, anchors.size, size=(n_text, G))]
+            x += np.float32(focus * gain) * bf16_bits_to_f32(L.k[b, h][pick])
+            q[b, :, h * G:(h + 1) * G] = x
+    return f32_to_bf16_bits(q), counts

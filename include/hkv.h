@@ -210,6 +210,30 @@ hkv_status hkv_allocate_budgets(int32_t n_heads, const uint8_t* head_type, const
                                 int64_t total_budget, double r, double alpha, uint32_t flags,
                                 int32_t* budgets_out);
 
+/* Text-centric head classification (Section 3.1, with the text-centric attention of Section 2.1):
+ * for every (sequence b, kv head h), S_text = softmax(Q_text K^T * scale) row by row over ALL C_b
+ * context tokens (no mask), the sum of each row's k_b = max(1, ceil(topk_fraction * C_b)) largest
+ * entries, and their mean over the rows: the text-centric sparsity score S in (0, 1].  A head is
+ * static (0) if S >= theta, else dynamic (1).  Under grouped-query attention the rows of a kv head
+ * are the text positions of every query head of its group (n_text[b] * G rows).
+ *   cfg          batch, n_q_heads, n_kv_heads, head_dim (128), max_seq_len, softmax_scale are read
+ *   k            dev bf16 [B, Hkv, max_seq_len, d]  keys of the prompt, as for hkv_compress
+ *   q_text       dev bf16 [B, n_text_max, Hq, d]    queries of the text tokens; rows >= n_text[b] are not read
+ *   seq_lens     host int32 [B]  C_b in 1..max_seq_len;   n_text  host int32 [B]  in 1..n_text_max
+ *   topk_fraction in (0, 1] (the paper's focus fraction is 0.05);  theta finite (the paper settles on 0.9)
+ *   workspace    dev, 256-B aligned, >= min_bytes of hkv_classify_workspace; with less than
+ *                preferred_bytes the rows are processed in several passes (same result)
+ *   scores_out   dev f64 [B, Hkv]  S (float32 softmax arithmetic, rows averaged in double, fixed order)
+ *   head_type_out dev u8 [B, Hkv]  the array hkv_plan / hkv_compress take, once copied to the host
+ * Enqueued on `stream`, no synchronisation; deterministic.  Errors: HKV_ERR_SHAPE (lengths),
+ * HKV_ERR_WORKSPACE, HKV_ERR_UNSUPPORTED (head_dim), HKV_ERR_INVALID_ARG. */
+hkv_status hkv_classify_workspace(const hkv_config* cfg, int32_t n_text_max, size_t* min_bytes,
+                                  size_t* preferred_bytes);
+hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, const void* q_text, int32_t n_text_max,
+                              const int32_t* seq_lens, const int32_t* n_text, double topk_fraction,
+                              double theta, void* workspace, size_t workspace_bytes, double* scores_out,
+                              uint8_t* head_type_out, void* stream);
+
 /* Chunk scoring + top-k for one dynamic head WITHOUT any caller- or library-allocated scratch.
  * (The paper has no counterpart: this is a packaging variant of the selection step of
  * hkv_select_chunks.)  It exists for callers that cannot allocate device memory where they call

@@ -27,7 +27,8 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_attend", "hkv_decode_attn_host", "hkv_cache_destroy",
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
-           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append", "hkv_decode_step_host"]
+           "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append", "hkv_decode_step_host",
+           "hkv_classify_workspace", "hkv_classify_heads"]
 
 
 class hkv_config(C.Structure):
@@ -83,6 +84,10 @@ def _load() -> C.CDLL:
     lib.hkv_decode_cluster_capacity.argtypes = [C.c_int32, i32p]
     lib.hkv_allocate_budgets.argtypes = [C.c_int32, u8p, C.POINTER(C.c_double), C.c_int64, C.c_double, C.c_double,
                                          C.c_uint32, i32p]
+    lib.hkv_classify_workspace.argtypes = [C.POINTER(hkv_config), C.c_int32, C.POINTER(C.c_size_t),
+                                           C.POINTER(C.c_size_t)]
+    lib.hkv_classify_heads.argtypes = [C.POINTER(hkv_config), vp, vp, C.c_int32, i32p, i32p, C.c_double, C.c_double,
+                                       vp, C.c_size_t, vp, vp, vp]
     lib.hkv_status_string.argtypes = [C.c_int]
     lib.hkv_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -279,6 +284,26 @@ def hkv_allocate_budgets(head_type, scores, total_budget: int, r: float, alpha: 
     _check(lib.hkv_allocate_budgets(ht.size, _ptr(ht, C.c_uint8), sp, int(total_budget), float(r), float(alpha),
                                     int(flags), _ptr(out, C.c_int32)), "hkv_allocate_budgets")
     return out
+
+
+def hkv_classify_workspace(cfg: hkv_config, n_text_max: int):
+    """(min_bytes, preferred_bytes) of the workspace hkv_classify_heads takes."""
+    lo, hi = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.hkv_classify_workspace(C.byref(cfg), int(n_text_max), C.byref(lo), C.byref(hi)),
+           "hkv_classify_workspace")
+    return int(lo.value), int(hi.value)
+
+
+def hkv_classify_heads(cfg: hkv_config, k, q_text, seq_lens, n_text, topk_fraction: float, theta: float,
+                       workspace, scores_out, head_type_out, stream=None):
+    """Text-centric sparsity score and static / dynamic label of every (sequence, kv head); see hkv.h.
+    k, q_text, workspace, scores_out (float64) and head_type_out (uint8) are CUDA tensors."""
+    sl, nt = _i32(seq_lens), _i32(n_text)
+    _check(lib.hkv_classify_heads(C.byref(cfg), k.data_ptr(), q_text.data_ptr(), int(q_text.shape[1]),
+                                  _ptr(sl, C.c_int32), _ptr(nt, C.c_int32), float(topk_fraction), float(theta),
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                  scores_out.data_ptr(), head_type_out.data_ptr(), _stream(stream)),
+           "hkv_classify_heads")
 
 
 def hkv_cache_stats(cache: int) -> dict:

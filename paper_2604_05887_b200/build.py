@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libhkv.so")
-SOURCES = ["hkv_api.cu", "hkv_compress.cu", "hkv_decode.cu", "hkv_noalloc.cu", "hkv_policy.cu"]
+SOURCES = ["hkv_api.cu", "hkv_classify.cu", "hkv_compress.cu", "hkv_decode.cu", "hkv_noalloc.cu", "hkv_policy.cu"]
 
 
 def _nvcc() -> str:

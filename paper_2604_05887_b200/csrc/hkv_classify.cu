@@ -1,0 +1,560 @@
+// Text-centric head classification (paper Section 3.1): for every (sequence, kv head) the rows of
+// S_text = softmax(Q_text K^T / sqrt(d)) over the whole context, the sum of each row's k largest
+// entries, their mean over the rows (the text-centric sparsity score) and the comparison with the
+// threshold theta.  Runs once per prompt and layer, before the budgets and the compression.
+//
+// Three kernels per pass over a block of rows:
+//   cls_logits_kernel  base-2 logits of a 64-key tile for the block's rows, tensor cores, float32
+//                      into the workspace;
+//   cls_row_kernel     one CTA per row: the row in shared memory, max, p = 2^(l - max), normaliser,
+//                      the exact k-th largest p (histogram over the float bits, then exact ranking
+//                      of the threshold bin), the sum of the entries above it plus the tied share;
+//   cls_finish_kernel  (after the last pass) mean of the rows' sums in double, fixed order, and
+//                      the label.
+#include <algorithm>
+#include <cmath>
+
+#include "hkv_device.cuh"
+#include "hkv_internal.h"
+
+namespace hkv {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kClsBatch = 64;          // sequences one group of launches takes
+constexpr int kClsTile = 64;           // key columns per CTA of the logits kernel
+constexpr int kClsWarps = 8;
+constexpr int kClsRowThreads = 1024;
+constexpr int kClsSmemCols = 49152;    // longest row the row kernel keeps in shared memory
+constexpr int kClsRank = 256;          // largest threshold bin that is sorted directly
+constexpr int kClsBins = 4096;          // bits 30..18 of a float in [0, 1]: 32 bins per octave
+constexpr int kClsShift = 18;
+constexpr int kClsLoadParts = 4;       // pieces a row arrives in, so that the maximum overlaps the copy
+constexpr int kClsRowScratch = (kClsBins + kClsRank + 32 + 8 + 32) * 4 + kClsLoadParts * 8;   // histogram, candidates, reduction slots, control words, warp sums, mbarriers
+
+struct ClsParams {
+  int32_t C[kClsBatch];   // context length of each sequence
+  int32_t T[kClsBatch];   // text tokens (query rows / group) of each sequence
+  int32_t k[kClsBatch];   // entries summed per row
+  int32_t n_kv_heads, n_q_heads, group, max_seq_len, t_stride;
+  int32_t row_begin, row_block;   // this pass covers rows [row_begin, row_begin + row_block) of every unit
+  int32_t c_stride;               // floats between two rows of the logits workspace (multiple of 64)
+  int32_t r_stride;               // floats between two units of the row-sum array
+  int32_t smem_cols;              // rows up to this length are staged in shared memory
+  float scale_log2e;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Logits.  One CTA = one 64-key tile of one unit; warps loop over the 16-row tiles of the pass.
+// Row r of a unit is (text token r / G, query head r % G of the group).
+// logits: float [unit][row_block][c_stride]
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kClsWarps * 32)
+    cls_logits_kernel(const ClsParams P, const __nv_bfloat16* kin, const __nv_bfloat16* q_text, float* logits) {
+  __shared__ __align__(128) uint8_t ktile[kClsTile * kRowBytes];
+  const int unit = blockIdx.y, b = unit / P.n_kv_heads, h = unit - b * P.n_kv_heads;
+  const int C = P.C[b], G = P.group, R = P.T[b] * G;
+  const int j0 = blockIdx.x * kClsTile;
+  if (j0 >= C || P.row_begin >= R) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+
+  const uint4* ksrc = reinterpret_cast<const uint4*>(
+      kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim);
+  for (int idx = tid; idx < kClsTile * 16; idx += kClsWarps * 32) {
+    const int row = idx >> 4, c = idx & 15;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (j0 + row < C) v = ksrc[static_cast<size_t>(j0 + row) * 16 + c];
+    *reinterpret_cast<uint4*>(ktile + row * kRowBytes + ((c ^ (row & 7)) << 4)) = v;
+  }
+  __syncthreads();
+
+  const uint32_t kbase = smem_u32(ktile);
+  const int mj = lane >> 3, mi = lane & 7;
+  const int krow = mi + ((mj >> 1) << 3), kcsel = mj & 1;
+  const int r_end = min(R, P.row_begin + P.row_block);
+  const int n_mt = (r_end - P.row_begin + 15) / 16;
+  float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride + j0;
+  for (int mt = warp; mt < n_mt; mt += kClsWarps) {
+    const int r0 = P.row_begin + mt * 16 + g, r1 = r0 + 8;
+    const int i0 = r0 / G, i1 = r1 / G;
+    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(
+        q_text + ((static_cast<size_t>(b) * P.t_stride + i0) * P.n_q_heads + h * G + (r0 - i0 * G)) * kHeadDim);
+    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(
+        q_text + ((static_cast<size_t>(b) * P.t_stride + i1) * P.n_q_heads + h * G + (r1 - i1 * G)) * kHeadDim);
+    uint32_t qa[8][4];
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      qa[kk][0] = (r0 < r_end) ? q0[kk * 8 + t] : 0u;
+      qa[kk][2] = (r0 < r_end) ? q0[kk * 8 + 4 + t] : 0u;
+      qa[kk][1] = (r1 < r_end) ? q1[kk * 8 + t] : 0u;
+      qa[kk][3] = (r1 < r_end) ? q1[kk * 8 + 4 + t] : 0u;
+    }
+    float s[8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < 4; ++sl) {
+      const int r = sl * 16 + krow;
+      const uint32_t rowaddr = kbase + r * kRowBytes;
+      const uint32_t key = r & 7;
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(b0, b1, b2, b3, rowaddr + (((2 * kk + kcsel) ^ key) << 4));
+        mma_bf16(s[2 * sl], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
+        mma_bf16(s[2 * sl + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+      }
+    }
+    float* o0 = out + static_cast<size_t>(r0 - P.row_begin) * P.c_stride + 2 * t;
+    float* o1 = out + static_cast<size_t>(r1 - P.row_begin) * P.c_stride + 2 * t;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      if (r0 < r_end)
+        *reinterpret_cast<float2*>(o0 + n * 8) = make_float2(s[n][0] * P.scale_log2e, s[n][1] * P.scale_log2e);
+      if (r1 < r_end)
+        *reinterpret_cast<float2*>(o1 + n * 8) = make_float2(s[n][2] * P.scale_log2e, s[n][3] * P.scale_log2e);
+    }
+  }
+}
+
+// Whole block (kClsRowThreads threads, every one calls): the highest bin b of hist[0, nbins) with
+// count(bins > b) < need <= count(bins >= b).  ctl[0] = b, ctl[1] = need - count(bins > b),
+// ctl[2] = count(b); visible after the caller's next barrier.  nbins is 4096, 1024 or 256; wsum is
+// scratch for 32 ints.
+__device__ __forceinline__ void cls_find_bin(const int* hist, int nbins, int need, int* ctl, int* wsum) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int loc[4] = {0, 0, 0, 0};
+  const int per = nbins == 4096 ? 4 : 1;
+  if (per == 4) {
+    const int4 v = reinterpret_cast<const int4*>(hist)[tid];
+    loc[0] = v.x; loc[1] = v.y; loc[2] = v.z; loc[3] = v.w;
+  } else if (tid < nbins) {
+    loc[0] = hist[tid];
+  }
+  const int tot = (loc[0] + loc[1]) + (loc[2] + loc[3]);
+  int run = tot;   // becomes the sum over this and the higher lanes of the warp
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_down_sync(0xffffffffu, run, off);
+    if (lane + off < 32) run += v;
+  }
+  if (lane == 0) wsum[warp] = run;
+  __syncthreads();
+  const int wt = wsum[lane];
+  int wrun = wt;   // sum over warps >= lane
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_down_sync(0xffffffffu, wrun, off);
+    if (lane + off < 32) wrun += v;
+  }
+  int acc = __shfl_sync(0xffffffffu, wrun - wt, warp) + run - tot;   // items in the bins above this thread's
+  if (acc < need && need <= acc + tot) {
+#pragma unroll
+    for (int j = 3; j >= 0; --j) {
+      if (j < per && acc < need && need <= acc + loc[j]) {
+        ctl[0] = tid * per + j;
+        ctl[1] = need - acc;
+        ctl[2] = loc[j];
+      }
+      if (j < per) acc += loc[j];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sum of the k largest softmax entries of every row; a persistent CTA takes one row at a time.
+// The row's logits arrive in shared memory by bulk copy (the next row is meanwhile prefetched into
+// L2) and are replaced by p = 2^(l - max) in [0, 1], whose float bits order like the values.  The
+// k-th largest p is found exactly: a histogram over bits 30..18 of p (32 bins per octave, so the
+// lanes of a warp rarely meet in a bin), then the threshold bin's entries are sorted outright (four
+// threads per entry) and the first `need` of them join the sum of everything above the bin; a
+// crowded bin is first narrowed by histograms over bits 17..8 and 7..0.  Sums run in a fixed
+// order, so the result is deterministic.
+// rowsum: float [unit][r_stride]
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kClsRowThreads)
+    cls_row_kernel(const ClsParams P, float* logits, float* rowsum, int rows_pass, int total_rows) {
+  extern __shared__ __align__(16) uint8_t cls_smem[];
+  int* hist = reinterpret_cast<int*>(cls_smem);                   // [kClsBins]
+  uint32_t* cand = reinterpret_cast<uint32_t*>(hist + kClsBins);  // [kClsRank]
+  float* red = reinterpret_cast<float*>(cand + kClsRank);         // [32]
+  int* ctl = reinterpret_cast<int*>(red + 32);                    // [8]
+  int* wsum = ctl + 8;                                            // [32]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(wsum + 32);         // [kClsLoadParts]
+  float* srow = reinterpret_cast<float*>(cls_smem + kClsRowScratch);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int i = 0; i < kClsLoadParts; ++i) mbar_init(bar + i, 1);
+    mbar_fence_init();
+  }
+  uint32_t phases = 0;   // bit i: parity the next wait on barrier i looks for
+
+  // block-wide reductions in a fixed order; every thread gets the result
+  auto block_sum = [&](float v) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    v = red[lane];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+  };
+  auto block_max = [&](float v) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    v = red[lane];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    return v;
+  };
+  // row `idx` of the pass: its unit, length and place; false for the rows a short sequence does not have
+  auto locate = [&](int idx, int* unit, int* C, int* r, size_t* off) {
+    if (idx >= total_rows) return false;
+    *unit = idx / rows_pass;
+    const int rr = idx - *unit * rows_pass, b = *unit / P.n_kv_heads;
+    *C = P.C[b];
+    *r = P.row_begin + rr;
+    *off = (static_cast<size_t>(*unit) * P.row_block + rr) * P.c_stride;
+    return *r < P.T[b] * P.group;
+  };
+
+  for (int idx = blockIdx.x; idx < total_rows; idx += gridDim.x) {
+    int unit, C, r;
+    size_t row_off;
+    if (!locate(idx, &unit, &C, &r, &row_off)) continue;
+    const int k = P.k[unit / P.n_kv_heads];
+    const bool staged = C <= P.smem_cols;
+    // p overwrites the logits: in shared memory, or for longer rows in place in the workspace
+    float* row = staged ? srow : logits + row_off;
+    float4* row4 = reinterpret_cast<float4*>(row);
+    const int n4 = (C + 3) >> 2;
+    // the row arrives in kClsLoadParts pieces of part4 float4s (a multiple of the block size), each on its own barrier
+    const int part4 = ((n4 + kClsLoadParts - 1) / kClsLoadParts + kClsRowThreads - 1) / kClsRowThreads * kClsRowThreads;
+
+    __syncthreads();   // the previous row's readers are done with the buffers
+    if (tid == 0 && staged) {
+      // whole 16-byte pieces: rows start 256-byte aligned and are padded to a multiple of 64 floats
+      fence_proxy_async();
+      for (int part = 0; part < kClsLoadParts; ++part) {
+        const int beg = part * part4, end = min(n4, beg + part4);
+        if (beg >= end) break;
+        mbar_arrive_expect_tx(bar + part, static_cast<uint32_t>(end - beg) * 16u);
+        for (int o = beg; o < end; o += 2048)
+          bulk_g2s(row4 + o, reinterpret_cast<const float4*>(logits + row_off) + o,
+                   static_cast<uint32_t>(min(2048, end - o)) * 16u, bar + part);
+      }
+      // start the next row's trip from HBM to L2 meanwhile
+      int u2, C2, r2;
+      size_t off2;
+      if (locate(idx + gridDim.x, &u2, &C2, &r2, &off2) && C2 <= P.smem_cols) {
+        const uint32_t b2 = static_cast<uint32_t>((C2 + 3) / 4 * 16);
+        for (uint32_t o = 0; o < b2; o += 32768u)
+          bulk_prefetch_l2(reinterpret_cast<const char*>(logits + off2) + o, min(32768u, b2 - o));
+      }
+    }
+    for (int i = tid; i < kClsBins; i += kClsRowThreads) hist[i] = 0;
+    if (tid == 0) ctl[3] = 0;
+
+    // maximum, piece by piece as the row lands; the up to three floats between C and the next
+    // multiple of four become -inf, that is p = 0: zeros below every real entry, which no top-k
+    // sum can feel
+    float mx = -INFINITY;
+    bool landed = true;
+    for (int part = 0; part < kClsLoadParts; ++part) {
+      const int beg = part * part4, end = min(n4, beg + part4);
+      if (beg >= end) break;
+      if (staged && landed) {
+        landed = mbar_wait_bounded(bar + part, (phases >> part) & 1u);
+        phases ^= 1u << part;
+      }
+      if (!landed) continue;
+      for (int i = beg + tid; i < end; i += kClsRowThreads) {
+        float4 v = row4[i];
+        if (i == n4 - 1 && (C & 3)) {
+          if ((C & 3) < 2) v.y = -INFINITY;
+          if ((C & 3) < 3) v.z = -INFINITY;
+          v.w = -INFINITY;
+          row4[i] = v;
+        }
+        mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+      }
+    }
+    if (__syncthreads_or(!landed)) {   // never seen; the whole CTA leaves, the row's sum and the score become NaN
+      if (tid == 0) rowsum[static_cast<size_t>(unit) * P.r_stride + r] = __int_as_float(0x7FC00000);
+      return;
+    }
+    const float M = block_max(mx);
+
+    // p, normaliser, histogram
+    auto prob = [&](float l) {
+      float q = fast_exp2(l - M);
+      if (!(q >= 0.f)) q = 0.f;      // a NaN logit counts as no attention
+      return fminf(q, 1.f);          // every bit pattern stays in [0, bits(1)]
+    };
+    float z = 0.f;
+    for (int i = tid; i < n4; i += kClsRowThreads) {
+      const float4 v = row4[i];
+      const float4 q = make_float4(prob(v.x), prob(v.y), prob(v.z), prob(v.w));
+      row4[i] = q;
+      z += (q.x + q.y) + (q.z + q.w);
+      atomicAdd(&hist[__float_as_uint(q.x) >> kClsShift], 1);
+      atomicAdd(&hist[__float_as_uint(q.y) >> kClsShift], 1);
+      atomicAdd(&hist[__float_as_uint(q.z) >> kClsShift], 1);
+      atomicAdd(&hist[__float_as_uint(q.w) >> kClsShift], 1);
+    }
+    const float Z = block_sum(z);   // its barriers also publish the histogram
+    cls_find_bin(hist, kClsBins, k, ctl, wsum);
+    __syncthreads();
+    uint32_t prefix = static_cast<uint32_t>(ctl[0]);
+    int shift = kClsShift, need = ctl[1], cnt = ctl[2];
+    float top = 0.f;
+    for (;;) {
+      if (need == cnt) {                      // the whole bin is inside the top k
+        for (int i = tid; i < n4; i += kClsRowThreads) {
+          const float4 q = row4[i];
+          top += (((__float_as_uint(q.x) >> shift) >= prefix ? q.x : 0.f) +
+                  ((__float_as_uint(q.y) >> shift) >= prefix ? q.y : 0.f)) +
+                 (((__float_as_uint(q.z) >> shift) >= prefix ? q.z : 0.f) +
+                  ((__float_as_uint(q.w) >> shift) >= prefix ? q.w : 0.f));
+        }
+        break;
+      }
+      if (cnt <= kClsRank) {
+        // sum what lies above the bin, collect the bin's entries (a warp that meets some reserves
+        // their slots with one atomic) and sort them exactly (descending; equal values in an
+        // arbitrary but complete order): the first `need` join the sum
+        for (int i0 = warp * 32; i0 < n4; i0 += kClsRowThreads) {
+          const int i = i0 + lane;
+          const float4 q = i < n4 ? row4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t hi = __float_as_uint(e[c]) >> shift;
+            if (hi > prefix) top += e[c];
+            const bool in_bin = i < n4 && hi == prefix;
+            const uint32_t m = __ballot_sync(0xffffffffu, in_bin);
+            if (m) {
+              int base = 0;
+              if (lane == 0) base = atomicAdd(&ctl[3], __popc(m));
+              base = __shfl_sync(0xffffffffu, base, 0);
+              if (in_bin) cand[base + __popc(m & ((1u << lane) - 1u))] = __float_as_uint(e[c]);
+            }
+          }
+        }
+        __syncthreads();
+        float* sorted = reinterpret_cast<float*>(hist);
+        const int c = tid >> 2, part = tid & 3;          // four threads rank one entry
+        int above = 0, before = 0;
+        const uint32_t mk = c < cnt ? cand[c] : 0u;
+        if (c < cnt) {
+          for (int j = part; j < cnt; j += 4) {
+            const uint32_t o = cand[j];
+            above += o > mk;
+            before += (o == mk) && (j < c);
+          }
+        }
+        above += __shfl_xor_sync(0xffffffffu, above, 1);
+        above += __shfl_xor_sync(0xffffffffu, above, 2);
+        before += __shfl_xor_sync(0xffffffffu, before, 1);
+        before += __shfl_xor_sync(0xffffffffu, before, 2);
+        if (c < cnt && part == 0) sorted[above + before] = __uint_as_float(mk);
+        __syncthreads();
+        if (tid < need) top += sorted[tid];
+        break;
+      }
+      if (shift == 0) {                       // more than kClsRank copies of one value: `need` of them count
+        for (int i = tid; i < n4; i += kClsRowThreads) {
+          const float4 q = row4[i];
+          top += ((__float_as_uint(q.x) > prefix ? q.x : 0.f) + (__float_as_uint(q.y) > prefix ? q.y : 0.f)) +
+                 ((__float_as_uint(q.z) > prefix ? q.z : 0.f) + (__float_as_uint(q.w) > prefix ? q.w : 0.f));
+        }
+        if (tid == 0) top += static_cast<float>(need) * __uint_as_float(prefix);
+        break;
+      }
+      // a crowded bin: histogram of the next bits of its entries (17..8, then 7..0)
+      const int width = shift == kClsShift ? 10 : 8;
+      const int nshift = shift - width;
+      const uint32_t mask = (1u << width) - 1u;
+      for (int i = tid; i < (1 << width); i += kClsRowThreads) hist[i] = 0;
+      __syncthreads();
+      auto count = [&](float q) {
+        const uint32_t u = __float_as_uint(q);
+        if ((u >> shift) == prefix) atomicAdd(&hist[(u >> nshift) & mask], 1);
+      };
+      for (int i = tid; i < n4; i += kClsRowThreads) {
+        const float4 q = row4[i];
+        count(q.x); count(q.y); count(q.z); count(q.w);
+      }
+      __syncthreads();
+      cls_find_bin(hist, 1 << width, need, ctl, wsum);
+      __syncthreads();
+      prefix = (prefix << width) | static_cast<uint32_t>(ctl[0]);
+      shift = nshift;
+      need = ctl[1];
+      cnt = ctl[2];
+    }
+    top = block_sum(top);
+    if (tid == 0) rowsum[static_cast<size_t>(unit) * P.r_stride + r] = top / Z;
+  }
+}
+
+// Mean of a unit's row sums (double, fixed order) and its label: 0 static if score >= theta, else 1.
+__global__ void __launch_bounds__(256)
+    cls_finish_kernel(const ClsParams P, const float* rowsum, double theta, double* scores_out, uint8_t* type_out,
+                      int unit0) {
+  __shared__ double part[256];
+  const int unit = blockIdx.x, b = unit / P.n_kv_heads;
+  const int R = P.T[b] * P.group;
+  const float* rs = rowsum + static_cast<size_t>(unit) * P.r_stride;
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < R; i += 256) acc += static_cast<double>(rs[i]);
+  part[threadIdx.x] = acc;
+  __syncthreads();
+  for (int s = 128; s >= 1; s >>= 1) {
+    if (threadIdx.x < s) part[threadIdx.x] += part[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double score = part[0] / static_cast<double>(R);
+    scores_out[unit0 + unit] = score;
+    type_out[unit0 + unit] = score >= theta ? 0 : 1;
+  }
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+hkv_status cls_check(const hkv_config* cfg, int32_t n_text_max) {
+  if (!cfg) return HKV_ERR_INVALID_ARG;
+  if (cfg->batch < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->max_seq_len < 1 || n_text_max < 1)
+    return HKV_ERR_SHAPE;
+  if (cfg->n_q_heads % cfg->n_kv_heads != 0) return HKV_ERR_SHAPE;
+  if (cfg->head_dim != kHeadDim || cfg->n_kv_heads > 60000 || cfg->max_seq_len > (1 << 23)) return HKV_ERR_UNSUPPORTED;
+  if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return HKV_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(n_text_max) * (cfg->n_q_heads / cfg->n_kv_heads) > (1 << 24)) return HKV_ERR_UNSUPPORTED;
+  return HKV_OK;
+}
+
+// sequences per group of launches, units of a group, bytes of the row-sum array in front of the logits
+struct ClsShape {
+  int group_batch, group_units, r_max;
+  size_t head_bytes;
+};
+ClsShape cls_shape(const hkv_config* cfg, int32_t n_text_max) {
+  ClsShape s;
+  s.group_batch = std::min(std::min(cfg->batch, kClsBatch), 60000 / cfg->n_kv_heads);
+  s.group_units = s.group_batch * cfg->n_kv_heads;
+  s.r_max = n_text_max * (cfg->n_q_heads / cfg->n_kv_heads);
+  s.head_bytes = round_up(static_cast<size_t>(s.group_units) * s.r_max * sizeof(float), kAlign);
+  return s;
+}
+
+}  // namespace
+
+}  // namespace hkv
+
+using namespace hkv;
+
+extern "C" hkv_status hkv_classify_workspace(const hkv_config* cfg, int32_t n_text_max, size_t* min_bytes,
+                                             size_t* preferred_bytes) {
+  const hkv_status st = cls_check(cfg, n_text_max);
+  if (st != HKV_OK) return st;
+  if (!min_bytes && !preferred_bytes) return HKV_ERR_INVALID_ARG;
+  const ClsShape s = cls_shape(cfg, n_text_max);
+  const size_t row_bytes = round_up(cfg->max_seq_len, kClsTile) * sizeof(float) * s.group_units;
+  if (min_bytes) *min_bytes = s.head_bytes + 16 * row_bytes;
+  if (preferred_bytes) {
+    // every row at once, up to half a gigabyte of logits
+    size_t rows = round_up(s.r_max, 16);
+    const size_t cap = std::max<size_t>(16, (static_cast<size_t>(512) << 20) / row_bytes / 16 * 16);
+    rows = std::min(rows, cap);
+    *preferred_bytes = s.head_bytes + rows * row_bytes;
+  }
+  return HKV_OK;
+}
+
+extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, const void* q_text,
+                                         int32_t n_text_max, const int32_t* seq_lens, const int32_t* n_text,
+                                         double topk_fraction, double theta, void* workspace,
+                                         size_t workspace_bytes, double* scores_out, uint8_t* head_type_out,
+                                         void* stream) {
+  const hkv_status st = cls_check(cfg, n_text_max);
+  if (st != HKV_OK) return st;
+  if (!k || !q_text || !seq_lens || !n_text || !workspace || !scores_out || !head_type_out)
+    return HKV_ERR_INVALID_ARG;
+  if (!(topk_fraction > 0.0 && topk_fraction <= 1.0) || !std::isfinite(theta)) return HKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return HKV_ERR_WORKSPACE;
+  int c_max = 0;
+  for (int b = 0; b < cfg->batch; ++b) {
+    if (seq_lens[b] < 1 || seq_lens[b] > cfg->max_seq_len) return HKV_ERR_SHAPE;
+    if (n_text[b] < 1 || n_text[b] > n_text_max) return HKV_ERR_SHAPE;
+    c_max = std::max(c_max, seq_lens[b]);
+  }
+  const ClsShape s = cls_shape(cfg, n_text_max);
+  const int G = cfg->n_q_heads / cfg->n_kv_heads;
+  const size_t c_stride = round_up(c_max, kClsTile);
+  const size_t row_bytes = c_stride * sizeof(float) * s.group_units;
+  if (workspace_bytes < s.head_bytes + 16 * row_bytes) return HKV_ERR_WORKSPACE;
+  const int row_block = static_cast<int>(
+      std::min<size_t>(round_up(s.r_max, 16), (workspace_bytes - s.head_bytes) / row_bytes / 16 * 16));
+
+  const int smem_cols = static_cast<int>(round_up(std::min(c_max, kClsSmemCols), kClsTile));
+  const size_t row_smem = kClsRowScratch + static_cast<size_t>(smem_cols) * sizeof(float);
+  if (cudaFuncSetAttribute(cls_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(row_smem)) != cudaSuccess)
+    return HKV_ERR_CUDA;
+
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
+    return HKV_ERR_CUDA;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  float* rowsum = static_cast<float*>(workspace);
+  float* logits = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.head_bytes);
+  const float scale =
+      cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(cfg->head_dim));
+  for (int b0 = 0; b0 < cfg->batch; b0 += s.group_batch) {
+    const int nb = std::min(s.group_batch, cfg->batch - b0);
+    ClsParams P{};
+    int r_max = 0, cg_max = 0;
+    for (int i = 0; i < nb; ++i) {
+      const int C = seq_lens[b0 + i];
+      P.C[i] = C;
+      P.T[i] = n_text[b0 + i];
+      const double kk = std::ceil(topk_fraction * static_cast<double>(C) - 1e-9);
+      P.k[i] = static_cast<int32_t>(std::max(1.0, std::min(static_cast<double>(C), kk)));
+      r_max = std::max(r_max, P.T[i] * G);
+      cg_max = std::max(cg_max, C);
+    }
+    P.n_kv_heads = cfg->n_kv_heads;
+    P.n_q_heads = cfg->n_q_heads;
+    P.group = G;
+    P.max_seq_len = cfg->max_seq_len;
+    P.t_stride = n_text_max;
+    P.row_block = row_block;
+    P.c_stride = static_cast<int32_t>(c_stride);
+    P.r_stride = s.r_max;
+    P.smem_cols = smem_cols;
+    P.scale_log2e = scale * kLog2e;
+    const __nv_bfloat16* kg = static_cast<const __nv_bfloat16*>(k) +
+                              static_cast<size_t>(b0) * cfg->n_kv_heads * cfg->max_seq_len * kHeadDim;
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(q_text) +
+                              static_cast<size_t>(b0) * n_text_max * cfg->n_q_heads * kHeadDim;
+    const int units = nb * cfg->n_kv_heads;
+    for (int rb = 0; rb < r_max; rb += row_block) {
+      P.row_begin = rb;
+      const int rows = std::min(row_block, r_max - rb);
+      cls_logits_kernel<<<dim3((cg_max + kClsTile - 1) / kClsTile, units), kClsWarps * 32, 0, cs>>>(P, kg, qg, logits);
+      const int total_rows = rows * units;
+      cls_row_kernel<<<std::min(total_rows, n_sm), kClsRowThreads, row_smem, cs>>>(P, logits, rowsum, rows, total_rows);
+    }
+    cls_finish_kernel<<<units, 256, 0, cs>>>(P, rowsum, theta, scores_out, head_type_out, b0 * cfg->n_kv_heads);
+    if (cudaGetLastError() != cudaSuccess) return HKV_ERR_CUDA;
+  }
+  return HKV_OK;
+}

@@ -59,3 +59,109 @@ def test_oracle_monotone_and_bounded():
         assert prev < s <= 1.0 + 1e-12 and s >= co.topk_count(C, f) / C - 1e-12
         prev = s
     assert co.classify(0.95, 0.9) == 0 and co.classify(0.9, 0.9) == 0 and co.classify(0.85, 0.9) == 1
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA path against the oracle
+# ---------------------------------------------------------------------------------------------
+SCORE_TOL = 1e-4     # float32 softmax arithmetic against float64
+
+
+def _oracle_scores(L, q_text, counts, fraction):
+    G = L.group
+    scale = 1.0 / math.sqrt(L.head_dim)
+    out = np.zeros((L.batch, L.n_kv_heads))
+    for b in range(L.batch):
+        C, T = int(L.seq_lens[b]), int(counts[b])
+        for h in range(L.n_kv_heads):
+            out[b, h] = co.sparsity_score(q_text[b, :T, h * G:(h + 1) * G], L.k[b, h, :C], scale, fraction)
+    return out
+
+
+def _gpu_scores(L, q_text, counts, fraction, theta, workspace="preferred"):
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import to_device_bf16
+    cfg = hkv.hkv_config(batch=L.batch, n_q_heads=L.n_q_heads, n_kv_heads=L.n_kv_heads, head_dim=L.head_dim,
+                         max_seq_len=L.max_seq_len, chunk_size=L.chunk_size, obs_window=L.obs_window,
+                         softmax_scale=0.0, flags=0, append_capacity=0)
+    lo, hi = hkv.hkv_classify_workspace(cfg, q_text.shape[1])
+    assert 0 < lo <= hi
+    ws = torch.empty(lo if workspace == "min" else hi, dtype=torch.uint8, device="cuda")
+    scores = torch.full((L.batch, L.n_kv_heads), -1.0, dtype=torch.float64, device="cuda")
+    types = torch.full((L.batch, L.n_kv_heads), 9, dtype=torch.uint8, device="cuda")
+    hkv.hkv_classify_heads(cfg, to_device_bf16(L.k), to_device_bf16(q_text), L.seq_lens, counts, fraction, theta,
+                           ws, scores, types)
+    torch.cuda.synchronize()
+    return scores.cpu().numpy(), types.cpu().numpy()
+
+
+def _check_case(L, n_text, fraction, theta=None, workspace="preferred", seed=5):
+    q_text, counts = hi.text_queries(L, n_text, seed=seed)
+    ref = _oracle_scores(L, q_text, counts, fraction)
+    if theta is None:
+        srt = np.sort(ref.ravel())
+        theta = float(0.5 * (srt[srt.size // 2 - 1] + srt[srt.size // 2])) if srt.size > 1 else 0.9
+    got, types = _gpu_scores(L, q_text, counts, fraction, theta, workspace)
+    err = np.abs(got - ref).max()
+    assert err <= SCORE_TOL, (err, got, ref)
+    for b in range(L.batch):
+        for h in range(L.n_kv_heads):
+            if abs(ref[b, h] - theta) > SCORE_TOL:
+                assert types[b, h] == co.classify(ref[b, h], theta), (b, h, ref[b, h], theta)
+            assert types[b, h] == (0 if got[b, h] >= theta else 1)
+    return ref, got
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("workspace", ["preferred", "min"])
+def test_gpu_classify_ragged_batch(workspace):
+    L = hi.tiny(seed=31, B=3, C=3000, chunk_size=32, w=8, Hq=28, Hkv=4, d=128)
+    ref, _ = _check_case(L, 20, 0.05, workspace=workspace)
+    assert ref.max() - ref.min() > 0.3            # the heads really span diffuse to peaked
+    _check_case(L, 20, 0.05, theta=0.9, workspace=workspace)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("fraction", [1e-6, 0.01, 0.5, 1.0])
+def test_gpu_classify_topk_counts(fraction):
+    L = hi.tiny(seed=32, B=2, C=1500, chunk_size=32, w=8, Hq=8, Hkv=2, d=128)
+    ref, got = _check_case(L, 9, fraction)
+    if fraction == 1.0:
+        assert np.abs(got - 1.0).max() < 1e-5
+
+
+@pytest.mark.gpu
+def test_gpu_classify_rows_longer_than_shared_memory():
+    L = hi.tiny(seed=33, B=1, C=50021, chunk_size=32, w=8, Hq=8, Hkv=2, d=128)
+    _check_case(L, 3, 0.05)
+
+
+@pytest.mark.gpu
+def test_gpu_classify_more_sequences_than_one_launch_group():
+    L = hi.tiny(seed=34, B=70, C=400, chunk_size=32, w=8, Hq=4, Hkv=2, d=128, ragged=False)
+    _check_case(L, 4, 0.05)
+
+
+@pytest.mark.gpu
+def test_gpu_classify_uniform_rows_and_errors():
+    from paper_2604_05887_b200 import binding as hkv
+    L = hi.tiny(seed=35, B=1, C=640, chunk_size=32, w=8, Hq=4, Hkv=2, d=128, ragged=False)
+    L.k[:] = L.k[:, :, :1]                         # identical keys: every row is uniform, score = k / C
+    q_text, counts = hi.text_queries(L, 5)
+    got, types = _gpu_scores(L, q_text, counts, 0.05, 0.9)
+    assert np.abs(got - 32 / 640).max() < 1e-6 and np.all(types == 1)
+    cfg = hkv.hkv_config(batch=1, n_q_heads=4, n_kv_heads=2, head_dim=128, max_seq_len=640, chunk_size=32,
+                         obs_window=8, softmax_scale=0.0, flags=0, append_capacity=0)
+    lo, _ = hkv.hkv_classify_workspace(cfg, 5)
+    ws = torch.empty(lo, dtype=torch.uint8, device="cuda")
+    sc = torch.zeros((1, 2), dtype=torch.float64, device="cuda")
+    ty = torch.zeros((1, 2), dtype=torch.uint8, device="cuda")
+    k = torch.zeros((1, 2, 640, 128), dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((1, 5, 4, 128), dtype=torch.bfloat16, device="cuda")
+    for kwargs, status in ((dict(seq_lens=[641]), 2), (dict(n_text=[6]), 2), (dict(n_text=[0]), 2),
+                           (dict(fraction=0.0), 1), (dict(fraction=1.5), 1), (dict(ws=ws[:lo - 256]), 4)):
+        a = dict(seq_lens=[640], n_text=[5], fraction=0.05, ws=ws)
+        a.update(kwargs)
+        with pytest.raises(hkv.HkvError) as e:
+            hkv.hkv_classify_heads(cfg, k, q, a["seq_lens"], a["n_text"], a["fraction"], 0.9, a["ws"], sc, ty)
+        assert e.value.status == status
