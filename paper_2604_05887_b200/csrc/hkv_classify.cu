@@ -4,8 +4,8 @@
 // threshold theta.  Runs once per prompt and layer, before the budgets and the compression.
 //
 // Three kernels per pass over a block of rows:
-//   cls_logits_kernel  base-2 logits of a 64-key tile for the block's rows, tensor cores, float32
-//                      into the workspace;
+//   cls_logits_tc_kernel  base-2 logits of 256 rows x a range of 128-key tiles, tcgen05 tensor cores,
+//                      float32 into the workspace (rows padded to a multiple of 128 floats);
 //   cls_row_kernel     one CTA per row: the row in shared memory, max, p = 2^(l - max), normaliser,
 //                      the exact k-th largest p (histogram over the float bits, then exact ranking
 //                      of the threshold bin), the sum of the entries above it plus the tied share;
@@ -16,6 +16,7 @@
 
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
+#include "hkv_tc.cuh"
 
 namespace hkv {
 
@@ -23,8 +24,6 @@ namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kClsBatch = 64;          // sequences one group of launches takes
-constexpr int kClsTile = 64;           // key columns per CTA of the logits kernel
-constexpr int kClsWarps = 8;
 constexpr int kClsRowThreads = 1024;
 constexpr int kClsSmemCols = 49152;    // longest row the row kernel keeps in shared memory
 constexpr int kClsRank = 256;          // largest threshold bin that is sorted directly
@@ -39,83 +38,69 @@ struct ClsParams {
   int32_t k[kClsBatch];   // entries summed per row
   int32_t n_kv_heads, n_q_heads, group, max_seq_len, t_stride;
   int32_t row_begin, row_block;   // this pass covers rows [row_begin, row_begin + row_block) of every unit
-  int32_t c_stride;               // floats between two rows of the logits workspace (multiple of 64)
+  int32_t c_stride;               // floats between two rows of the logits workspace (multiple of 128)
   int32_t r_stride;               // floats between two units of the row-sum array
   int32_t smem_cols;              // rows up to this length are staged in shared memory
   float scale_log2e;
 };
 
 // ---------------------------------------------------------------------------------------------
-// Logits.  One CTA = one 64-key tile of one unit; warps loop over the 16-row tiles of the pass.
-// Row r of a unit is (text token r / G, query head r % G of the group).
-// logits: float [unit][row_block][c_stride]
+// Logits (tcgen05 tensor cores, accumulators in tensor memory).  One CTA = 256 rows of one unit (two accumulator blocks) x a range of
+// 128-key tiles; a draining thread owns one row of each block and writes its 128 logits of the tile
+// as 512 contiguous bytes.  grid (key ranges, 256-row blocks of the pass, units).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kClsWarps * 32)
-    cls_logits_kernel(const ClsParams P, const __nv_bfloat16* kin, const __nv_bfloat16* q_text, float* logits) {
-  __shared__ __align__(128) uint8_t ktile[kClsTile * kRowBytes];
-  const int unit = blockIdx.y, b = unit / P.n_kv_heads, h = unit - b * P.n_kv_heads;
+__global__ void __launch_bounds__(tc::kThreads, 1)
+    cls_logits_tc_kernel(const ClsParams P, const __nv_bfloat16* kin, const __nv_bfloat16* q_text, float* logits,
+                         int tiles_per_cta, int32_t* err) {
+  extern __shared__ __align__(16) uint8_t tc_smem[];
+  const int unit = blockIdx.z, b = unit / P.n_kv_heads, h = unit - b * P.n_kv_heads;
   const int C = P.C[b], G = P.group, R = P.T[b] * G;
-  const int j0 = blockIdx.x * kClsTile;
-  if (j0 >= C || P.row_begin >= R) return;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-
-  const uint4* ksrc = reinterpret_cast<const uint4*>(
-      kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim);
-  for (int idx = tid; idx < kClsTile * 16; idx += kClsWarps * 32) {
-    const int row = idx >> 4, c = idx & 15;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (j0 + row < C) v = ksrc[static_cast<size_t>(j0 + row) * 16 + c];
-    *reinterpret_cast<uint4*>(ktile + row * kRowBytes + ((c ^ (row & 7)) << 4)) = v;
-  }
-  __syncthreads();
-
-  const uint32_t kbase = smem_u32(ktile);
-  const int mj = lane >> 3, mi = lane & 7;
-  const int krow = mi + ((mj >> 1) << 3), kcsel = mj & 1;
   const int r_end = min(R, P.row_begin + P.row_block);
-  const int n_mt = (r_end - P.row_begin + 15) / 16;
-  float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride + j0;
-  for (int mt = warp; mt < n_mt; mt += kClsWarps) {
-    const int r0 = P.row_begin + mt * 16 + g, r1 = r0 + 8;
-    const int i0 = r0 / G, i1 = r1 / G;
-    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(
-        q_text + ((static_cast<size_t>(b) * P.t_stride + i0) * P.n_q_heads + h * G + (r0 - i0 * G)) * kHeadDim);
-    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(
-        q_text + ((static_cast<size_t>(b) * P.t_stride + i1) * P.n_q_heads + h * G + (r1 - i1 * G)) * kHeadDim);
-    uint32_t qa[8][4];
+  const int row0 = P.row_begin + blockIdx.y * tc::kQRows;
+  const int n_tiles = (C + tc::kKeysPerTile - 1) / tc::kKeysPerTile;
+  const int tile_begin = blockIdx.x * tiles_per_cta, tile_end = min(n_tiles, tile_begin + tiles_per_cta);
+  if (row0 >= r_end || tile_begin >= tile_end) return;
+
+  auto q_row = [&](int row) -> const __nv_bfloat16* {
+    const int r = row0 + row;
+    if (r >= r_end) return nullptr;
+    const int i = r / G;
+    return q_text + ((static_cast<size_t>(b) * P.t_stride + i) * P.n_q_heads + h * G + (r - i * G)) * kHeadDim;
+  };
+  const __nv_bfloat16* keys =
+      kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim;
+  float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride;
+  const float sc = P.scale_log2e;
+  auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch) {
+    // accumulator columns 128 half .. + 127 are the tile's keys for rows row0 + 128 half + (0..127)
+    const int rbase = row0 + 128 * half + (lane_row & ~31);   // first row of this warp
+    if (rbase >= r_end) return;                               // the warp's rows are all padding
+    const int lane = lane_row & 31;
+    float* dst = out + static_cast<size_t>(rbase - P.row_begin) * P.c_stride +
+                 static_cast<size_t>(tile) * tc::kKeysPerTile;
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+      float v[32];
+      load(g, v);
+      // through the scratch (16-byte pieces XOR-permuted by the row) so that the global stores are
+      // whole 128-byte runs of one row: 8 lanes per row, 4 rows per instruction
+      float4* mine = reinterpret_cast<float4*>(scratch + lane * 32);
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      qa[kk][0] = (r0 < r_end) ? q0[kk * 8 + t] : 0u;
-      qa[kk][2] = (r0 < r_end) ? q0[kk * 8 + 4 + t] : 0u;
-      qa[kk][1] = (r1 < r_end) ? q1[kk * 8 + t] : 0u;
-      qa[kk][3] = (r1 < r_end) ? q1[kk * 8 + 4 + t] : 0u;
-    }
-    float s[8][4];
+      for (int c = 0; c < 8; ++c)
+        mine[c ^ (lane & 7)] = make_float4(v[4 * c] * sc, v[4 * c + 1] * sc, v[4 * c + 2] * sc, v[4 * c + 3] * sc);
+      __syncwarp();
 #pragma unroll
-    for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-#pragma unroll
-    for (int sl = 0; sl < 4; ++sl) {
-      const int r = sl * 16 + krow;
-      const uint32_t rowaddr = kbase + r * kRowBytes;
-      const uint32_t key = r & 7;
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(b0, b1, b2, b3, rowaddr + (((2 * kk + kcsel) ^ key) << 4));
-        mma_bf16(s[2 * sl], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
-        mma_bf16(s[2 * sl + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+      for (int it = 0; it < 8; ++it) {
+        const int rr = it * 4 + (lane >> 3), c = lane & 7;
+        const float4 val = reinterpret_cast<const float4*>(scratch + rr * 32)[c ^ (rr & 7)];
+        if (rbase + rr < r_end)
+          *reinterpret_cast<float4*>(dst + static_cast<size_t>(rr) * P.c_stride + g * 32 + c * 4) = val;
       }
+      __syncwarp();
     }
-    float* o0 = out + static_cast<size_t>(r0 - P.row_begin) * P.c_stride + 2 * t;
-    float* o1 = out + static_cast<size_t>(r1 - P.row_begin) * P.c_stride + 2 * t;
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      if (r0 < r_end)
-        *reinterpret_cast<float2*>(o0 + n * 8) = make_float2(s[n][0] * P.scale_log2e, s[n][1] * P.scale_log2e);
-      if (r1 < r_end)
-        *reinterpret_cast<float2*>(o1 + n * 8) = make_float2(s[n][2] * P.scale_log2e, s[n][3] * P.scale_log2e);
-    }
-  }
+  };
+  if (!tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue) && threadIdx.x == 0)
+    atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT);
 }
 
 // Whole block (kClsRowThreads threads, every one calls): the highest bin b of hist[0, nbins) with
@@ -239,7 +224,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
 
     __syncthreads();   // the previous row's readers are done with the buffers
     if (tid == 0 && staged) {
-      // whole 16-byte pieces: rows start 256-byte aligned and are padded to a multiple of 64 floats
+      // whole 16-byte pieces: rows start 256-byte aligned and are padded to a multiple of 128 floats
       fence_proxy_async();
       for (int part = 0; part < kClsLoadParts; ++part) {
         const int beg = part * part4, end = min(n4, beg + part4);
@@ -406,8 +391,8 @@ __global__ void __launch_bounds__(kClsRowThreads)
 
 // Mean of a unit's row sums (double, fixed order) and its label: 0 static if score >= theta, else 1.
 __global__ void __launch_bounds__(256)
-    cls_finish_kernel(const ClsParams P, const float* rowsum, double theta, double* scores_out, uint8_t* type_out,
-                      int unit0) {
+    cls_finish_kernel(const ClsParams P, const float* rowsum, const int32_t* err, double theta, double* scores_out,
+                      uint8_t* type_out, int unit0) {
   __shared__ double part[256];
   const int unit = blockIdx.x, b = unit / P.n_kv_heads;
   const int R = P.T[b] * P.group;
@@ -421,7 +406,8 @@ __global__ void __launch_bounds__(256)
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const double score = part[0] / static_cast<double>(R);
+    // a device-side wait that ran out (never seen) turns every score into NaN
+    const double score = err[0] == 0 ? part[0] / static_cast<double>(R) : __longlong_as_double(0x7FF8000000000000ll);
     scores_out[unit0 + unit] = score;
     type_out[unit0 + unit] = score >= theta ? 0 : 1;
   }
@@ -443,14 +429,14 @@ hkv_status cls_check(const hkv_config* cfg, int32_t n_text_max) {
 // sequences per group of launches, units of a group, bytes of the row-sum array in front of the logits
 struct ClsShape {
   int group_batch, group_units, r_max;
-  size_t head_bytes;
+  size_t head_bytes;   // error word (kAlign bytes) + row sums
 };
 ClsShape cls_shape(const hkv_config* cfg, int32_t n_text_max) {
   ClsShape s;
   s.group_batch = std::min(std::min(cfg->batch, kClsBatch), 60000 / cfg->n_kv_heads);
   s.group_units = s.group_batch * cfg->n_kv_heads;
   s.r_max = n_text_max * (cfg->n_q_heads / cfg->n_kv_heads);
-  s.head_bytes = round_up(static_cast<size_t>(s.group_units) * s.r_max * sizeof(float), kAlign);
+  s.head_bytes = kAlign + round_up(static_cast<size_t>(s.group_units) * s.r_max * sizeof(float), kAlign);
   return s;
 }
 
@@ -466,7 +452,7 @@ extern "C" hkv_status hkv_classify_workspace(const hkv_config* cfg, int32_t n_te
   if (st != HKV_OK) return st;
   if (!min_bytes && !preferred_bytes) return HKV_ERR_INVALID_ARG;
   const ClsShape s = cls_shape(cfg, n_text_max);
-  const size_t row_bytes = round_up(cfg->max_seq_len, kClsTile) * sizeof(float) * s.group_units;
+  const size_t row_bytes = round_up(cfg->max_seq_len, tc::kKeysPerTile) * sizeof(float) * s.group_units;
   if (min_bytes) *min_bytes = s.head_bytes + 16 * row_bytes;
   if (preferred_bytes) {
     // every row at once, up to half a gigabyte of logits
@@ -497,13 +483,13 @@ extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, c
   }
   const ClsShape s = cls_shape(cfg, n_text_max);
   const int G = cfg->n_q_heads / cfg->n_kv_heads;
-  const size_t c_stride = round_up(c_max, kClsTile);
+  const size_t c_stride = round_up(c_max, tc::kKeysPerTile);
   const size_t row_bytes = c_stride * sizeof(float) * s.group_units;
   if (workspace_bytes < s.head_bytes + 16 * row_bytes) return HKV_ERR_WORKSPACE;
   const int row_block = static_cast<int>(
       std::min<size_t>(round_up(s.r_max, 16), (workspace_bytes - s.head_bytes) / row_bytes / 16 * 16));
 
-  const int smem_cols = static_cast<int>(round_up(std::min(c_max, kClsSmemCols), kClsTile));
+  const int smem_cols = static_cast<int>(round_up(std::min(c_max, kClsSmemCols), 64));
   const size_t row_smem = kClsRowScratch + static_cast<size_t>(smem_cols) * sizeof(float);
   if (cudaFuncSetAttribute(cls_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            static_cast<int>(row_smem)) != cudaSuccess)
@@ -514,7 +500,12 @@ extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, c
       cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
     return HKV_ERR_CUDA;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  float* rowsum = static_cast<float*>(workspace);
+  int32_t* err = static_cast<int32_t*>(workspace);
+  float* rowsum = reinterpret_cast<float*>(static_cast<char*>(workspace) + kAlign);
+  if (cudaMemsetAsync(err, 0, kAlign, cs) != cudaSuccess) return HKV_ERR_CUDA;
+  if (cudaFuncSetAttribute(cls_logits_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) !=
+      cudaSuccess)
+    return HKV_ERR_CUDA;
   float* logits = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.head_bytes);
   const float scale =
       cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(cfg->head_dim));
@@ -549,11 +540,17 @@ extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, c
     for (int rb = 0; rb < r_max; rb += row_block) {
       P.row_begin = rb;
       const int rows = std::min(row_block, r_max - rb);
-      cls_logits_kernel<<<dim3((cg_max + kClsTile - 1) / kClsTile, units), kClsWarps * 32, 0, cs>>>(P, kg, qg, logits);
+      // key ranges sized so that the launch is about one wave of CTAs
+      const int row_blocks = (rows + tc::kQRows - 1) / tc::kQRows;
+      const int n_tiles = (cg_max + tc::kKeysPerTile - 1) / tc::kKeysPerTile;
+      const int splits = std::max(1, std::min(n_tiles, n_sm / std::max(1, units * row_blocks)));
+      const int tiles_per_cta = (n_tiles + splits - 1) / splits;
+      cls_logits_tc_kernel<<<dim3((n_tiles + tiles_per_cta - 1) / tiles_per_cta, row_blocks, units), tc::kThreads,
+                             tc::kSmemBytes, cs>>>(P, kg, qg, logits, tiles_per_cta, err);
       const int total_rows = rows * units;
       cls_row_kernel<<<std::min(total_rows, n_sm), kClsRowThreads, row_smem, cs>>>(P, logits, rowsum, rows, total_rows);
     }
-    cls_finish_kernel<<<units, 256, 0, cs>>>(P, rowsum, theta, scores_out, head_type_out, b0 * cfg->n_kv_heads);
+    cls_finish_kernel<<<units, 256, 0, cs>>>(P, rowsum, err, theta, scores_out, head_type_out, b0 * cfg->n_kv_heads);
     if (cudaGetLastError() != cudaSuccess) return HKV_ERR_CUDA;
   }
   return HKV_OK;
