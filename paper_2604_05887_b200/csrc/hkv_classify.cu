@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim;
   float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride;
   const float sc = P.scale_log2e;
-  auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch) {
+  auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch, float*, uint64_t*) {
     // accumulator columns 128 half .. + 127 are the tile's keys for rows row0 + 128 half + (0..127)
     const int rbase = row0 + 128 * half + (lane_row & ~31);   // first row of this warp
     if (rbase >= r_end) return;                               // the warp's rows are all padding

@@ -3,16 +3,17 @@
 // the chunk means plus the copy of K/V into the cache.  K/V rows are written with their sixteen
 // 16-byte pieces XOR-permuted by (row & 7), the layout the flash-decode kernel stages with plain
 // bulk copies and reads with bank-conflict-free ldmatrix.
+#include <algorithm>
+
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
+#include "hkv_tc.cuh"
 
 namespace hkv {
 
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kWsTile = 64;      // key columns per CTA of the window-score kernels
-constexpr int kWsWarps = 8;
 
 __device__ __forceinline__ const Unit* unit_of(const char* cache, const Header* hdr, bool dynamic, int ordinal,
                                                int* uid_out) {
@@ -23,165 +24,149 @@ __device__ __forceinline__ const Unit* unit_of(const char* cache, const Header* 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Window scores.  S_w = softmax over ALL tokens of the w*G window rows' logits, s_w = mean of rows.
-// MODE 0: per (row, column tile) running max and exp-sum.  MODE 1: with the rows' final (max, sum)
-// known, column sums of the normalised probabilities -> s_w.
-// One CTA = one 64-token column tile of one static unit; warps loop over 16-row tiles of the
-// R = w*G rows; logits on tensor cores.
-// stats: float2 [n_static][n_tiles_max][Rpad], final: float2 [n_static][Rpad]
+// Window scores.  S_w = softmax over ALL tokens of the w*G window rows' logits, s_w = mean of rows
+// (row r = window position r / G, query head r % G of the group).  The logits run on the tcgen05
+// tensor cores: one CTA = one static unit x one range of 128-key tiles x one block of up to 256
+// rows; the row block stays in shared memory, the key tiles stream; logits in base 2.
+// MODE 0: accumulator rows = window rows; a draining thread owns one row and keeps its running
+//         (max, exp-sum) over the CTA's keys; stats: float2 [n_static][n_ranges_max][Rpad].
+// MODE 1: with the rows' final (max, sum) known, accumulator rows = keys; a draining thread owns
+//         one key and sums the normalised probabilities of its half of the rows, the two halves
+//         meet in shared memory, and s_w[key] (+)= sum / R (written by the first row block, added
+//         to by later ones).
+// grid (key ranges, n_static).
 // ---------------------------------------------------------------------------------------------
 template <int MODE>
-__global__ void __launch_bounds__(kWsWarps * 32)
-    window_scores_kernel(const char* cache, char* workspace, const __nv_bfloat16* kin, const __nv_bfloat16* q_obs,
-                         float2* stats, const float2* final_stats, int n_tiles_max, int Rpad) {
-  __shared__ __align__(128) uint8_t ktile[kWsTile * kRowBytes];
-  __shared__ float colsum[kWsWarps][kWsTile];
+__global__ void __launch_bounds__(tc::kThreads, 1)
+    window_scores_tc_kernel(char* cache, char* workspace, const __nv_bfloat16* kin, const __nv_bfloat16* q_obs,
+                            float2* stats, const float2* final_stats, int n_ranges_max, int Rpad,
+                            int tiles_per_cta, int row_block) {
+  extern __shared__ __align__(16) uint8_t tc_smem[];
+  __shared__ float4 rowinfo[tc::kQRows];   // MODE 1: (max, 1 / sum, last visible key, -) of each resident row
 
   const Header* hdr = reinterpret_cast<const Header*>(cache);
   const Unit* u = unit_of(cache, hdr, false, blockIdx.y, nullptr);
-  const int C = u->C, j0 = blockIdx.x * kWsTile;
-  if (j0 >= C) return;
-  const int G = hdr->group, w = hdr->obs_window, Hq = hdr->n_q_heads, Hkv = hdr->n_kv_heads;
-  const int R = w * G;
+  const int C = u->C, G = hdr->group, w = hdr->obs_window, Hq = hdr->n_q_heads, Hkv = hdr->n_kv_heads;
+  const int R = w * G, row0 = row_block * tc::kQRows;
+  const int n_tiles = (C + tc::kKeysPerTile - 1) / tc::kKeysPerTile;
+  const int tile_begin = blockIdx.x * tiles_per_cta, tile_end = min(n_tiles, tile_begin + tiles_per_cta);
+  if (tile_begin >= tile_end) return;
   const bool causal = (hdr->flags & HKV_CAUSAL_WINDOW) != 0;
   const float sc = hdr->scale * kLog2e;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int ub = u->b, uh = u->h;
 
-  // stage the key tile (rows past C are zero), 16-byte pieces permuted by row & 7
-  const uint4* ksrc = reinterpret_cast<const uint4*>(
-      kin + (static_cast<size_t>(u->b) * Hkv + u->h) * static_cast<size_t>(hdr->max_seq_len) * kHeadDim);
-  for (int idx = tid; idx < kWsTile * 16; idx += kWsWarps * 32) {
-    const int row = idx >> 4, c = idx & 15;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (j0 + row < C) v = ksrc[static_cast<size_t>(j0 + row) * 16 + c];
-    *reinterpret_cast<uint4*>(ktile + row * kRowBytes + ((c ^ (row & 7)) << 4)) = v;
-  }
-  __syncthreads();
+  auto q_row = [&](int row) -> const __nv_bfloat16* {
+    const int r = row0 + row;
+    if (r >= R) return nullptr;
+    const int i = r / G;
+    return q_obs + ((static_cast<size_t>(ub) * w + i) * Hq + uh * G + (r - i * G)) * kHeadDim;
+  };
+  const __nv_bfloat16* keys =
+      kin + (static_cast<size_t>(ub) * Hkv + uh) * static_cast<size_t>(hdr->max_seq_len) * kHeadDim;
+  int32_t* err = reinterpret_cast<int32_t*>(cache + hdr->err_off);
 
-  const uint32_t kbase = smem_u32(ktile);
-  const int mj = lane >> 3, mi = lane & 7;
-  const int krow = mi + ((mj >> 1) << 3), kcsel = mj & 1;
-  float cacc[8][2];
+  if (MODE == 0) {
+    float m_run = -INFINITY, z_run = 0.f;
+    int my_row = -1;
+    auto epilogue = [&](int tile, int lane_row, int half, auto load, float*, float*, uint64_t*) {
+      const int r = row0 + 128 * half + lane_row;
+      my_row = r;
+      if (row0 + 128 * half + (lane_row & ~31) >= R) return;   // the warp's rows are all padding
+      const int lim = causal ? (C - w + r / G) : (C - 1);      // last key the row sees
+      const int j0 = tile * tc::kKeysPerTile;
+#pragma unroll 1
+      for (int g = 0; g < 4; ++g) {
+        float v[32];
+        load(g, v);
+        const int jg = j0 + g * 32;
+        float gmax = -INFINITY;
 #pragma unroll
-  for (int n = 0; n < 8; ++n) cacc[n][0] = cacc[n][1] = 0.f;
-
-  const int n_mt = (R + 15) / 16;
-  for (int mt = warp; mt < n_mt; mt += kWsWarps) {
-    const int r0 = mt * 16 + g, r1 = r0 + 8;
-    const int i0 = r0 / G, i1 = r1 / G;   // window row index of each mma row
-    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(
-        q_obs + ((static_cast<size_t>(u->b) * w + i0) * Hq + u->h * G + (r0 - i0 * G)) * kHeadDim);
-    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(
-        q_obs + ((static_cast<size_t>(u->b) * w + i1) * Hq + u->h * G + (r1 - i1 * G)) * kHeadDim);
-    uint32_t qa[8][4];
+        for (int c = 0; c < 32; ++c) {
+          v[c] = (jg + c <= lim && jg + c < C) ? v[c] * sc : -INFINITY;
+          gmax = fmaxf(gmax, v[c]);
+        }
+        if (gmax > -INFINITY) {
+          const float m_new = fmaxf(m_run, gmax);
+          float acc = 0.f;
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      qa[kk][0] = (r0 < R) ? q0[kk * 8 + t] : 0u;
-      qa[kk][2] = (r0 < R) ? q0[kk * 8 + 4 + t] : 0u;
-      qa[kk][1] = (r1 < R) ? q1[kk * 8 + t] : 0u;
-      qa[kk][3] = (r1 < R) ? q1[kk * 8 + 4 + t] : 0u;
+          for (int c = 0; c < 32; ++c) acc += fast_exp2(v[c] - m_new);
+          z_run = z_run * fast_exp2(m_run - m_new) + acc;   // 2^(-inf) = 0 on the first visible group
+          m_run = m_new;
+        }
+      }
+    };
+    const bool ok = tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue);
+    if (threadIdx.x >= 64 && my_row >= 0 && my_row < R)
+      stats[(static_cast<size_t>(blockIdx.y) * n_ranges_max + blockIdx.x) * Rpad + my_row] = make_float2(m_run, z_run);
+    if (!ok && threadIdx.x == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrScoreWait; }
+  } else {
+    for (int i = threadIdx.x; i < tc::kQRows; i += tc::kThreads) {
+      const int r = row0 + i;
+      float4 info = make_float4(0.f, 0.f, -1.f, 0.f);   // a padding row sees no key
+      if (r < R) {
+        const float2 f = final_stats[static_cast<size_t>(blockIdx.y) * Rpad + r];
+        info = make_float4(f.x, 1.f / f.y, static_cast<float>(causal ? (C - w + r / G) : (C - 1)), 0.f);
+      }
+      rowinfo[i] = info;
     }
-    float s[8][4];
+    // (scores_cta synchronises the CTA before any tile is drained)
+    float* sw = reinterpret_cast<float*>(workspace + u->ws_scores_off);
+    const float inv_R = 1.f / static_cast<float>(R);
+    int n_done = 0;
+    bool pair_ok = true;
+    auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch, float* partner,
+                        uint64_t* pair_bar) {
+      const int j = tile * tc::kKeysPerTile + lane_row;
+      const float jf = static_cast<float>(j);
+      float acc = 0.f;
+      if (row0 + 128 * half < R) {                     // same for the whole warp
+#pragma unroll 1
+        for (int g = 0; g < 4; ++g) {
+          float v[32];
+          load(g, v);
+          const float4* info = rowinfo + 128 * half + 32 * g;
 #pragma unroll
-    for (int n = 0; n < 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-#pragma unroll
-    for (int sl = 0; sl < 4; ++sl) {
-      const int r = sl * 16 + krow;
-      const uint32_t rowaddr = kbase + r * kRowBytes;
-      const uint32_t key = r & 7;
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(b0, b1, b2, b3, rowaddr + (((2 * kk + kcsel) ^ key) << 4));
-        mma_bf16(s[2 * sl], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
-        mma_bf16(s[2 * sl + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+          for (int c = 0; c < 32; ++c) {
+            const float4 ri = info[c];
+            const float p = fast_exp2(fmaf(v[c], sc, -ri.x)) * ri.y;
+            acc += (jf <= ri.z) ? p : 0.f;
+          }
+        }
       }
-    }
-    // scale (base-2 logits) and mask: columns past C, and keys after the row's own position if causal
-    const int lim0 = causal ? (C - w + i0) : (C - 1), lim1 = causal ? (C - w + i1) : (C - 1);
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int j = j0 + n * 8 + 2 * t + e;
-        s[n][e] = (j < C && j <= lim0) ? s[n][e] * sc : -INFINITY;
-        s[n][2 + e] = (j < C && j <= lim1) ? s[n][2 + e] * sc : -INFINITY;
+      // the half-1 warp hands its sums over (two buffers, by tile parity); the half-0 warp adds and
+      // stores.  pair_bar is the barrier of this tile's parity: its (n_done / 2)-th use.
+      const int slot = (n_done & 1) * 32 + (lane_row & 31);
+      if (half == 1) {
+        scratch[slot] = acc;
+        tc::mbar_arrive(pair_bar);
+      } else {
+        if (pair_ok) pair_ok = mbar_wait_bounded(pair_bar, (n_done >> 1) & 1);
+        if (pair_ok && j < C) {
+          const float tot = (acc + partner[slot]) * inv_R;
+          sw[j] = row_block == 0 ? tot : sw[j] + tot;
+        }
       }
-    }
-    if (MODE == 0) {
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-      for (int n = 0; n < 8; ++n) {
-        mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
-        mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
-      }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      float z0 = 0.f, z1 = 0.f;
-      if (mx0 > -INFINITY) {
-#pragma unroll
-        for (int n = 0; n < 8; ++n) z0 += exp2f(s[n][0] - mx0) + exp2f(s[n][1] - mx0);
-      }
-      if (mx1 > -INFINITY) {
-#pragma unroll
-        for (int n = 0; n < 8; ++n) z1 += exp2f(s[n][2] - mx1) + exp2f(s[n][3] - mx1);
-      }
-      z0 += __shfl_xor_sync(0xffffffffu, z0, 1);
-      z0 += __shfl_xor_sync(0xffffffffu, z0, 2);
-      z1 += __shfl_xor_sync(0xffffffffu, z1, 1);
-      z1 += __shfl_xor_sync(0xffffffffu, z1, 2);
-      if (t == 0) {
-        float2* dst = stats + (static_cast<size_t>(blockIdx.y) * n_tiles_max + blockIdx.x) * Rpad;
-        if (r0 < R) dst[r0] = make_float2(mx0, z0);
-        if (r1 < R) dst[r1] = make_float2(mx1, z1);
-      }
-    } else {
-      const float2* fin = final_stats + static_cast<size_t>(blockIdx.y) * Rpad;
-      const float2 f0 = (r0 < R) ? fin[r0] : make_float2(0.f, 1.f);
-      const float2 f1 = (r1 < R) ? fin[r1] : make_float2(0.f, 1.f);
-      const float inv0 = (r0 < R) ? 1.f / f0.y : 0.f, inv1 = (r1 < R) ? 1.f / f1.y : 0.f;
-#pragma unroll
-      for (int n = 0; n < 8; ++n) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e)
-          cacc[n][e] += exp2f(s[n][e] - f0.x) * inv0 + exp2f(s[n][2 + e] - f1.x) * inv1;
-      }
-    }
-  }
-  if (MODE == 1) {
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        float v = cacc[n][e];
-        v += __shfl_xor_sync(0xffffffffu, v, 4);
-        v += __shfl_xor_sync(0xffffffffu, v, 8);
-        v += __shfl_xor_sync(0xffffffffu, v, 16);
-        if (g == 0) colsum[warp][n * 8 + 2 * t + e] = v;
-      }
-    }
-    __syncthreads();
-    if (tid < kWsTile && j0 + tid < C) {
-      float tot = 0.f;
-#pragma unroll
-      for (int w2 = 0; w2 < kWsWarps; ++w2) tot += colsum[w2][tid];
-      float* sw = reinterpret_cast<float*>(workspace + u->ws_scores_off);
-      sw[j0 + tid] = tot / static_cast<float>(R);
+      ++n_done;
+    };
+    const bool ok = tc::scores_cta<true>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue);
+    const bool pairs = __syncthreads_and(pair_ok);
+    if (!(ok && pairs) && threadIdx.x == 0) {
+      atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT);
+      err[1] = kErrScoreWait;
     }
   }
 }
 
-// Combines the per-tile (max, sum) of every window row into the row's final (max, sum): one warp per
-// row, lanes stride the column tiles.
+// Combines the per-range (max, sum) of every window row into the row's final (max, sum): one warp per
+// row, lanes stride the key ranges.
 constexpr int kRowReduceWarps = 8;
 __global__ void __launch_bounds__(kRowReduceWarps * 32)
-    window_rowreduce_kernel(const char* cache, const float2* stats, float2* final_stats, int n_tiles_max, int Rpad) {
+    window_rowreduce_kernel(const char* cache, const float2* stats, float2* final_stats, int n_tiles_max, int Rpad,
+                            int tiles_per_cta) {
   const Header* hdr = reinterpret_cast<const Header*>(cache);
   const Unit* u = unit_of(cache, hdr, false, blockIdx.y, nullptr);
   const int R = hdr->obs_window * hdr->group;
-  const int n_tiles = (u->C + kWsTile - 1) / kWsTile;
+  const int n_tiles = ((u->C + tc::kKeysPerTile - 1) / tc::kKeysPerTile + tiles_per_cta - 1) / tiles_per_cta;
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * kRowReduceWarps + (threadIdx.x >> 5);
   if (r >= R) return;
@@ -400,15 +385,31 @@ cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, co
   const int Rpad = (R + 15) / 16 * 16;
   float2* stats = reinterpret_cast<float2*>(workspace + ws_rowstat_off);
   float2* fin = stats + static_cast<size_t>(hdr.n_static) * n_col_tiles_max * Rpad;
-  dim3 grid(n_col_tiles_max, hdr.n_static);
-  window_scores_kernel<0><<<grid, kWsWarps * 32, 0, stream>>>(
-      cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
-      n_col_tiles_max, Rpad);
-  window_rowreduce_kernel<<<dim3((R + kRowReduceWarps - 1) / kRowReduceWarps, hdr.n_static), kRowReduceWarps * 32, 0, stream>>>(
-      cache, stats, fin, n_col_tiles_max, Rpad);
-  window_scores_kernel<1><<<grid, kWsWarps * 32, 0, stream>>>(
-      cache, workspace, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(q_obs), stats, fin,
-      n_col_tiles_max, Rpad);
+  int dev = 0, n_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(window_scores_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(window_scores_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  // key ranges sized so that one launch is at most one wave of CTAs; n_col_tiles_max counts 64-key tiles
+  const int n_tiles = (n_col_tiles_max + 1) / 2;
+  const int splits = std::max(1, std::min(n_tiles, n_sm / hdr.n_static));
+  const int tiles_per_cta = (n_tiles + splits - 1) / splits;
+  const int n_ranges = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+  const int n_row_blocks = (R + tc::kQRows - 1) / tc::kQRows;
+  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q_obs);
+  const dim3 grid(n_ranges, hdr.n_static);
+  for (int rb = 0; rb < n_row_blocks; ++rb)
+    window_scores_tc_kernel<0><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(cache, workspace, kb, qb, stats, fin,
+                                                                              n_col_tiles_max, Rpad, tiles_per_cta, rb);
+  window_rowreduce_kernel<<<dim3((R + kRowReduceWarps - 1) / kRowReduceWarps, hdr.n_static), kRowReduceWarps * 32, 0,
+                            stream>>>(cache, stats, fin, n_col_tiles_max, Rpad, tiles_per_cta);
+  for (int rb = 0; rb < n_row_blocks; ++rb)
+    window_scores_tc_kernel<1><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(cache, workspace, kb, qb, stats, fin,
+                                                                              n_col_tiles_max, Rpad, tiles_per_cta, rb);
   return cudaGetLastError();
 }
 

@@ -31,7 +31,7 @@ constexpr int kLoadLag = 2;                         // key tiles in flight per C
 constexpr int kTmemCols = 512;                      // two accumulator buffers of 256 columns
 constexpr int kDrainWarps = 8;                      // two per lane quarter: columns 0..127 and 128..255
 constexpr int kThreads = (2 + kDrainWarps) * 32;    // warp 0 loads, warp 1 issues, warps 2..9 drain
-constexpr int kBarBytes = 128;
+constexpr int kBarBytes = 256;
 constexpr int kScratchPerWarp = 4096;               // 32 x 32 floats a draining warp may use to reorder its output
 constexpr int kSmemBytes =
     kQBytes + kStages * kStageBytes + kDrainWarps * kScratchPerWarp + kBarBytes + 1024;   // + slack to align to 1024
@@ -122,10 +122,14 @@ __device__ __forceinline__ uint32_t piece_offset(int row, int piece, int plane_b
 //               columns 128 t .. 128 t + 127 = the tile's keys); true: accumulator rows = the tile's keys,
 //               columns = the 256 query rows
 //   epilogue    functor called by each of the 256 draining threads for every tile:
-//               epilogue(tile, lane 0..127, half 0..1, load, scratch): the thread owns accumulator lane
+//               epilogue(tile, lane 0..127, half 0..1, load, scratch, partner, pair_bar): the thread owns accumulator lane
 //               `lane`, columns 128 half .. 128 half + 127; load(g, v) reads its columns
 //               128 half + 32 g .. + 31 (g = 0..3) into float v[32] and must be called by whole warps;
-//               scratch is the warp's 4 KB of shared memory
+//               scratch is the warp's 4 KB of shared memory; partner is the scratch of the warp that owns
+//               the other column half of the same lanes, pair_bar a barrier (32 arrivals per phase;
+//               one for the even and one for the odd tiles of the CTA, so its k-th use has parity k & 1)
+//               the half-1 warp may use to hand data to the half-0 warp: the two accumulator buffers keep
+//               the warps within one tile of each other, so a phase is never met twice
 // Returns false if a bounded wait ran out (the caller reports it); tensor memory is freed either way.
 // ---------------------------------------------------------------------------------------------
 template <bool kKeysAsRows, class QRowFn, class Epilogue>
@@ -139,7 +143,8 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
   uint64_t* empty = full + kStages;
   uint64_t* acc_full = empty + kStages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* pair_bar = acc_empty + 2;   // [4][2]: per lane quarter, one for even and one for odd tiles
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pair_bar + 8);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_tiles = tile_end - tile_begin;
 
@@ -160,6 +165,7 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
       mbar_init(acc_full + b, 1);
       mbar_init(acc_empty + b, kDrainWarps * 32);
     }
+    for (int q = 0; q < 8; ++q) mbar_init(pair_bar + q, 32);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -240,7 +246,9 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
           tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * 256 + half * 128);
       epilogue(tile_begin + i, row, half,
                [&](int g, float (&v)[32]) { tmem_ld32(taddr + static_cast<uint32_t>(g * 32), v); },
-               reinterpret_cast<float*>(scratch + (warp - 2) * kScratchPerWarp));
+               reinterpret_cast<float*>(scratch + (warp - 2) * kScratchPerWarp),
+               reinterpret_cast<float*>(scratch + ((warp - 2) ^ 4) * kScratchPerWarp),
+               pair_bar + 2 * quarter + (i & 1));
       fence_before_sync();
       mbar_arrive(acc_empty + buf);
     }
