@@ -71,17 +71,14 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim;
   float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride;
   const float sc = P.scale_log2e;
-  auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch, float*, uint64_t*) {
+  auto epilogue = [&](int tile, int lane_row, int half, auto groups, float* scratch, float*, uint64_t*) {
     // accumulator columns 128 half .. + 127 are the tile's keys for rows row0 + 128 half + (0..127)
     const int rbase = row0 + 128 * half + (lane_row & ~31);   // first row of this warp
     if (rbase >= r_end) return;                               // the warp's rows are all padding
     const int lane = lane_row & 31;
     float* dst = out + static_cast<size_t>(rbase - P.row_begin) * P.c_stride +
                  static_cast<size_t>(tile) * tc::kKeysPerTile;
-#pragma unroll 1
-    for (int g = 0; g < 4; ++g) {
-      float v[32];
-      load(g, v);
+    groups([&](int g, float (&v)[32]) {
       // through the scratch (16-byte pieces XOR-permuted by the row) so that the global stores are
       // whole 128-byte runs of one row: 8 lanes per row, 4 rows per instruction
       float4* mine = reinterpret_cast<float4*>(scratch + lane * 32);
@@ -97,7 +94,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
           *reinterpret_cast<float4*>(dst + static_cast<size_t>(rr) * P.c_stride + g * 32 + c * 4) = val;
       }
       __syncwarp();
-    }
+    });
   };
   if (!tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue) && threadIdx.x == 0)
     atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT);

@@ -68,32 +68,39 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
   if (MODE == 0) {
     float m_run = -INFINITY, z_run = 0.f;
     int my_row = -1;
-    auto epilogue = [&](int tile, int lane_row, int half, auto load, float*, float*, uint64_t*) {
+    auto epilogue = [&](int tile, int lane_row, int half, auto groups, float*, float*, uint64_t*) {
       const int r = row0 + 128 * half + lane_row;
       my_row = r;
       if (row0 + 128 * half + (lane_row & ~31) >= R) return;   // the warp's rows are all padding
       const int lim = causal ? (C - w + r / G) : (C - 1);      // last key the row sees
       const int j0 = tile * tc::kKeysPerTile;
-#pragma unroll 1
-      for (int g = 0; g < 4; ++g) {
-        float v[32];
-        load(g, v);
+      const bool all_visible = j0 + tc::kKeysPerTile - 1 <= (causal ? C - w : C - 1);   // to every row
+      groups([&](int g, float (&v)[32]) {
         const int jg = j0 + g * 32;
         float gmax = -INFINITY;
+        if (all_visible) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          v[c] = (jg + c <= lim && jg + c < C) ? v[c] * sc : -INFINITY;
-          gmax = fmaxf(gmax, v[c]);
+          for (int c = 0; c < 32; ++c) gmax = fmaxf(gmax, v[c]);
+          gmax *= sc;   // the scale is positive
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            v[c] = (jg + c <= lim && jg + c < C) ? v[c] : -INFINITY;
+            gmax = fmaxf(gmax, v[c] * sc);
+          }
         }
         if (gmax > -INFINITY) {
           const float m_new = fmaxf(m_run, gmax);
-          float acc = 0.f;
+          float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-          for (int c = 0; c < 32; ++c) acc += fast_exp2(v[c] - m_new);
-          z_run = z_run * fast_exp2(m_run - m_new) + acc;   // 2^(-inf) = 0 on the first visible group
+          for (int c = 0; c < 32; c += 2) {
+            a0 += fast_exp2(fmaf(v[c], sc, -m_new));
+            a1 += fast_exp2(fmaf(v[c + 1], sc, -m_new));
+          }
+          z_run = z_run * fast_exp2(m_run - m_new) + (a0 + a1);   // 2^(-inf) = 0 on the first visible group
           m_run = m_new;
         }
-      }
+      });
     };
     const bool ok = tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue);
     if (threadIdx.x >= 64 && my_row >= 0 && my_row < R)
@@ -114,25 +121,33 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
     const float inv_R = 1.f / static_cast<float>(R);
     int n_done = 0;
     bool pair_ok = true;
-    auto epilogue = [&](int tile, int lane_row, int half, auto load, float* scratch, float* partner,
+    auto epilogue = [&](int tile, int lane_row, int half, auto groups, float* scratch, float* partner,
                         uint64_t* pair_bar) {
-      const int j = tile * tc::kKeysPerTile + lane_row;
+      const int j0 = tile * tc::kKeysPerTile, j = j0 + lane_row;
       const float jf = static_cast<float>(j);
-      float acc = 0.f;
+      const bool all_visible = j0 + tc::kKeysPerTile - 1 <= (causal ? C - w : C - 1);   // to every row
+      float acc = 0.f, acc2 = 0.f;
       if (row0 + 128 * half < R) {                     // same for the whole warp
-#pragma unroll 1
-        for (int g = 0; g < 4; ++g) {
-          float v[32];
-          load(g, v);
+        groups([&](int g, float (&v)[32]) {
           const float4* info = rowinfo + 128 * half + 32 * g;
+          if (all_visible) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float4 ri = info[c];
-            const float p = fast_exp2(fmaf(v[c], sc, -ri.x)) * ri.y;
-            acc += (jf <= ri.z) ? p : 0.f;
+            for (int c = 0; c < 32; c += 2) {
+              const float4 r0 = info[c], r1 = info[c + 1];   // a padding row has 1 / sum = 0
+              acc = fmaf(fast_exp2(fmaf(v[c], sc, -r0.x)), r0.y, acc);
+              acc2 = fmaf(fast_exp2(fmaf(v[c + 1], sc, -r1.x)), r1.y, acc2);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float4 ri = info[c];
+              const float p = fast_exp2(fmaf(v[c], sc, -ri.x)) * ri.y;
+              acc += (jf <= ri.z) ? p : 0.f;
+            }
           }
-        }
+        });
       }
+      acc += acc2;
       // the half-1 warp hands its sums over (two buffers, by tile parity); the half-0 warp adds and
       // stores.  pair_bar is the barrier of this tile's parity: its (n_done / 2)-th use.
       const int slot = (n_done & 1) * 32 + (lane_row & 31);

@@ -43,6 +43,9 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src, uint32_t 
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(src_bytes)
                : "memory");
 }
+__device__ __forceinline__ void cp_async16_addr(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -82,9 +85,9 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// 32 lanes x 32 consecutive columns: thread i of the warp gets lane (base lane + i), v[j] = column base + j
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 lanes x 32 consecutive columns: thread i of the warp gets lane (base lane + i), r[j] = column base + j.
+// The registers hold the values only after tmem_ld_wait(r), which also ties them to the wait for the compiler.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -94,9 +97,43 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+// The four 32-column groups of a draining thread's 128 columns, the read of group g + 1 in flight
+// while fn(g, v) works on group g.  Whole warps call it.
+template <class Fn>
+__device__ __forceinline__ void drain_groups(uint32_t taddr, Fn fn) {
+  uint32_t ra[32], rb[32];
+  float v[32];
+  tmem_ld32_issue(taddr, ra);
+  tmem_ld_wait(ra);
+  tmem_ld32_issue(taddr + 32u, rb);
 #pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
+  fn(0, v);
+  tmem_ld_wait(rb);
+  tmem_ld32_issue(taddr + 64u, ra);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rb[i]);
+  fn(1, v);
+  tmem_ld_wait(ra);
+  tmem_ld32_issue(taddr + 96u, rb);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
+  fn(2, v);
+  tmem_ld_wait(rb);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rb[i]);
+  fn(3, v);
 }
 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -123,8 +160,8 @@ __device__ __forceinline__ uint32_t piece_offset(int row, int piece, int plane_b
 //               columns = the 256 query rows
 //   epilogue    functor called by each of the 256 draining threads for every tile:
 //               epilogue(tile, lane 0..127, half 0..1, load, scratch, partner, pair_bar): the thread owns accumulator lane
-//               `lane`, columns 128 half .. 128 half + 127; load(g, v) reads its columns
-//               128 half + 32 g .. + 31 (g = 0..3) into float v[32] and must be called by whole warps;
+//               `lane`, columns 128 half .. 128 half + 127; groups(fn) calls fn(g, v) for g = 0..3 with its
+//               columns 128 half + 32 g .. + 31 in float v[32] and must be called by whole warps (or not at all);
 //               scratch is the warp's 4 KB of shared memory; partner is the scratch of the warp that owns
 //               the other column half of the same lanes, pair_bar a barrier (32 arrivals per phase;
 //               one for the even and one for the odd tiles of the CTA, so its k-th use has parity k & 1)
@@ -148,13 +185,23 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_tiles = tile_end - tile_begin;
 
-  // query block -> shared memory (plain loads and stores), barriers, tensor memory
-  for (int idx = tid; idx < kQRows * 16; idx += kThreads) {
-    const int row = idx >> 4, piece = idx & 15;
-    const __nv_bfloat16* src = q_row(row);
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (src) v = reinterpret_cast<const uint4*>(src)[piece];
-    *reinterpret_cast<uint4*>(qs + piece_offset(row, piece, kPlaneBytesQ)) = v;
+  // query block -> shared memory (plain loads, four in flight per thread, and stores), barriers, tensor memory
+  for (int base = tid; base < kQRows * 16; base += 4 * kThreads) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = base + u * kThreads;
+      v[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (idx < kQRows * 16) {
+        const __nv_bfloat16* src = q_row(idx >> 4);
+        if (src) v[u] = __ldg(reinterpret_cast<const uint4*>(src) + (idx & 15));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = base + u * kThreads;
+      if (idx < kQRows * 16) *reinterpret_cast<uint4*>(qs + piece_offset(idx >> 4, idx & 15, kPlaneBytesQ)) = v[u];
+    }
   }
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -181,18 +228,38 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
 
   if (warp == 0) {
     // ---- loader: 16-byte asynchronous copies, kLoadLag tiles ahead of the tile handed over ----
+    uint32_t ld_dst[4];
+    int ld_src[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int row = 2 * u + (lane >> 4), piece = lane & 15;
+      ld_dst[u] = piece_offset(row, piece, kPlaneBytesK);
+      ld_src[u] = row * 256 + piece * 16;
+    }
     for (int i = 0; i < n_tiles + kLoadLag; ++i) {
       if (i < n_tiles) {
         const int s = i % kStages;
         if (i >= kStages && !mbar_wait_bounded(empty + s, ((i / kStages) - 1) & 1)) { ok = false; break; }
         uint8_t* dst = ks + s * kStageBytes;
         const int j0 = (tile_begin + i) * kKeysPerTile;
+        if (j0 + kKeysPerTile <= C) {
+          // a whole tile: lane = (row parity r0, piece); rows 8 it + 2 u + r0, so the swizzle depends on u only
+          const uint32_t dbase = smem_u32(dst);
+          const char* sbase = reinterpret_cast<const char*>(keys + static_cast<size_t>(j0) * 128);
 #pragma unroll 4
-        for (int it = 0; it < kKeysPerTile * 16 / 32; ++it) {
-          const int p = it * 32 + lane, row = p >> 4, piece = p & 15;
-          const bool in = j0 + row < C;
-          const __nv_bfloat16* src = keys + static_cast<size_t>(in ? j0 + row : 0) * 128 + piece * 8;
-          cp_async16(dst + piece_offset(row, piece, kPlaneBytesK), src, in ? 16u : 0u);
+          for (int it = 0; it < kKeysPerTile / 8; ++it) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              cp_async16_addr(dbase + ld_dst[u] + static_cast<uint32_t>(it * 1024), sbase + ld_src[u] + it * 2048);
+          }
+        } else {
+#pragma unroll 4
+          for (int it = 0; it < kKeysPerTile * 16 / 32; ++it) {
+            const int p = it * 32 + lane, row = p >> 4, piece = p & 15;
+            const bool in = j0 + row < C;
+            const __nv_bfloat16* src = keys + static_cast<size_t>(in ? j0 + row : 0) * 128 + piece * 8;
+            cp_async16(dst + piece_offset(row, piece, kPlaneBytesK), src, in ? 16u : 0u);
+          }
         }
       }
       cp_async_commit();
@@ -244,8 +311,7 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
       fence_after_sync();
       const uint32_t taddr =
           tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * 256 + half * 128);
-      epilogue(tile_begin + i, row, half,
-               [&](int g, float (&v)[32]) { tmem_ld32(taddr + static_cast<uint32_t>(g * 32), v); },
+      epilogue(tile_begin + i, row, half, [&](auto fn) { drain_groups(taddr, fn); },
                reinterpret_cast<float*>(scratch + (warp - 2) * kScratchPerWarp),
                reinterpret_cast<float*>(scratch + ((warp - 2) ^ 4) * kScratchPerWarp),
                pair_bar + 2 * quarter + (i & 1));
