@@ -377,6 +377,15 @@ def main():
         outs.append(lc.new_out())
         if layer == 0:
             L0 = L
+            # compression proper: layer 0 again, after the allocator has seen these sizes once
+            comp_ms = []
+            for _ in range(4):
+                e0.record()
+                lc2 = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
+                e1.record()
+                torch.cuda.synchronize()
+                comp_ms.append(e0.elapsed_time(e1))
+                lc2.close()
         else:
             del L
         del k_dev, v_dev
@@ -493,7 +502,10 @@ def main():
                    "l2": "inputs larger than L2: one step streams %.0f MB of distinct KV" % (algo_bytes / 1e6)
                    if algo_bytes > 2 * 126e6 else "WARNING: step working set near L2 size",
                    "launch": "CUDA graph of one hkv_decode_attn per layer, layers in sequence",
-                   "compress_GBps_of_input_kv": kv_in_bytes / t_comp / 1e9},
+                   "compress_GBps_of_input_kv": kv_in_bytes / t_comp / 1e9,
+                   "compress_ms_per_layer": min(comp_ms),
+                   "compress_how": "hkv_compress of layer 0 repeated 4 times, fastest (the GB/s figure beside it "
+                                   "spans every layer's first compression, device allocations included)"},
         "frac_of_measured_peak": value / world / peak, "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "decode_kernel (score + top-k + flash-decode + merge, one launch per layer)",
                      "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",

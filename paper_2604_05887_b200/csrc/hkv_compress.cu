@@ -204,14 +204,20 @@ __global__ void __launch_bounds__(kRowReduceWarps * 32)
 // Static keep-set: window U text-before-window U Top-M visual-before-window by score (ties to the
 // lower position); when window + text exceed the budget, text is ranked instead; when the budget
 // does not exceed the window, the last `budget` tokens.  One CTA per static unit, ascending output.
+// The selection makes several passes over the tokens; each token's role (kept regardless / out of the
+// ranking / ranked by this key) is therefore computed once into shared memory.
 // ---------------------------------------------------------------------------------------------
 constexpr int kKeepThreads = 1024;
 constexpr int kKeepScratchInts = keyed_scratch_ints(kKeepThreads);
 
+constexpr uint32_t kKeepAlways = 0xFFFFFFFFu;   // no float's key (it would be a NaN's)
+
 __global__ void __launch_bounds__(kKeepThreads)
-    static_select_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text) {
+    static_select_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text,
+                         int key_slots) {
   __shared__ __align__(16) int scratch[kKeepScratchInts];
   __shared__ int s_ntext;
+  extern __shared__ __align__(16) uint32_t skey[];   // key_slots entries: every token's role, computed once
 
   const Header* hdr = reinterpret_cast<const Header*>(cache);
   int uid;
@@ -224,11 +230,17 @@ __global__ void __launch_bounds__(kKeepThreads)
                             : reinterpret_cast<const float*>(workspace + u->ws_scores_off);
   int32_t* out = reinterpret_cast<int32_t*>(cache + u->idx_off);
   const int hist_end = C - w;   // tokens before the window
+  const bool cached = C <= key_slots;
 
   if (tid == 0) s_ntext = 0;
   __syncthreads();
   int cnt = 0;
-  for (int i = tid; i < hist_end; i += kKeepThreads) cnt += txt[i] != 0;
+#pragma unroll 16
+  for (int i = tid; i < hist_end; i += kKeepThreads) {
+    const int t = txt[i] != 0;
+    cnt += t;
+    if (cached) skey[i] = static_cast<uint32_t>(t);
+  }
   for (int off = 16; off >= 1; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
   if ((tid & 31) == 0 && cnt) atomicAdd(&s_ntext, cnt);
   __syncthreads();
@@ -243,15 +255,33 @@ __global__ void __launch_bounds__(kKeepThreads)
     const int room = budget - w;
     const bool rank_text = n_text >= room;       // window + text do not fit: rank the text tokens
     const int k = rank_text ? room : room - n_text;
-    emitted = block_topk_keyed<kKeepThreads>(
-        C, k,
-        [&](int i) {
-          if (i >= hist_end) return 0u;
-          const bool is_t = txt[i] != 0;
-          return (is_t == rank_text) ? float_key(scores[i]) : 0u;
-        },
-        [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, [&](int pos, int i) { out[pos] = i; },
-        scratch);
+    if (cached) {
+      // each token's role once: kKeepAlways = kept regardless, 0 = out of the ranking, else its score's key
+      // (a thread rewrites only the entries it flagged above)
+#pragma unroll 16
+      for (int i = tid; i < C; i += kKeepThreads) {
+        uint32_t key = kKeepAlways;
+        if (i < hist_end) {
+          const bool is_t = skey[i] != 0u;
+          key = (is_t == rank_text) ? float_key(scores[i]) : (is_t ? kKeepAlways : 0u);
+        }
+        skey[i] = key;
+      }
+      __syncthreads();
+      emitted = block_topk_keyed<kKeepThreads>(
+          C, k, [&](int i) { const uint32_t v = skey[i]; return v == kKeepAlways ? 0u : v; },
+          [&](int i) { return skey[i] == kKeepAlways; }, [&](int pos, int i) { out[pos] = i; }, scratch);
+    } else {
+      emitted = block_topk_keyed<kKeepThreads>(
+          C, k,
+          [&](int i) {
+            if (i >= hist_end) return 0u;
+            const bool is_t = txt[i] != 0;
+            return (is_t == rank_text) ? float_key(scores[i]) : 0u;
+          },
+          [&](int i) { return i >= hist_end || (!rank_text && txt[i] != 0); }, [&](int pos, int i) { out[pos] = i; },
+          scratch);
+    }
   }
   if (tid == 0) {
     reinterpret_cast<int32_t*>(cache + hdr->n_valid_off)[uid] = emitted;
@@ -431,7 +461,14 @@ cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, co
 cudaError_t launch_static_select(char* cache, char* workspace, const float* token_scores, const uint8_t* is_text,
                                  const Header& hdr, cudaStream_t stream) {
   if (hdr.n_static == 0) return cudaSuccess;
-  static_select_kernel<<<hdr.n_static, kKeepThreads, 0, stream>>>(cache, workspace, token_scores, is_text);
+  // every token's role is kept in shared memory when the longest sequence fits (else it is recomputed per pass)
+  const int key_slots = std::min(hdr.max_seq_len, 49152);
+  const size_t smem = static_cast<size_t>(key_slots) * sizeof(uint32_t);
+  cudaError_t e =
+      cudaFuncSetAttribute(static_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  static_select_kernel<<<hdr.n_static, kKeepThreads, smem, stream>>>(cache, workspace, token_scores, is_text,
+                                                                     key_slots);
   return cudaGetLastError();
 }
 

@@ -436,37 +436,34 @@ __device__ int block_topk_keyed(int n, int k, KeyFn key, AlwaysFn always, EmitFn
     if (kv != 0u) atomicAdd(&hist[bin_of(kv)], 1);
   }
   __syncthreads();
-  // every warp: the highest bin b with count(bins > b) < k <= count(bins >= b); lane owns 32 bins
+  // the highest bin b with count(bins > b) < k <= count(bins >= b): thread t owns bin t, suffix sums by
+  // warp shuffles and one exchange of warp totals
   int tbin, need, cnt;
   {
-    int loc[32], tot = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int4 v = reinterpret_cast<const int4*>(hist)[lane * 8 + j];
-      loc[4 * j] = v.x; loc[4 * j + 1] = v.y; loc[4 * j + 2] = v.z; loc[4 * j + 3] = v.w;
-      tot += v.x + v.y + v.z + v.w;
-    }
-    int run = tot;
+    static_assert(NTHR == kKeyedBins, "one bin per thread");
+    const int mine = hist[tid];
+    int run = mine;   // becomes the sum over this and the higher lanes of the warp
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
       const int v = __shfl_down_sync(0xffffffffu, run, off);
       if (lane + off < 32) run += v;
     }
-    const int above = run - tot;
-    const bool mine = above < k && k <= above + tot;
-    int my_bin = 0, my_need = 0, my_cnt = 0;
-    if (mine) {
-      int acc = above;
+    if (lane == 0) wtot[warp] = run;
+    __syncthreads();
+    const int wt = wtot[lane];
+    int wrun = wt;    // sum over warps >= lane
 #pragma unroll
-      for (int j = 31; j >= 0; --j) {
-        if (acc < k && k <= acc + loc[j]) { my_bin = lane * 32 + j; my_need = k - acc; my_cnt = loc[j]; }
-        acc += loc[j];
-      }
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_down_sync(0xffffffffu, wrun, off);
+      if (lane + off < 32) wrun += v;
     }
-    const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
-    tbin = __shfl_sync(0xffffffffu, my_bin, src);
-    need = __shfl_sync(0xffffffffu, my_need, src);
-    cnt = __shfl_sync(0xffffffffu, my_cnt, src);
+    const int above = __shfl_sync(0xffffffffu, wrun - wt, warp) + run - mine;
+    if (above < k && k <= above + mine) { misc[1] = tid; misc[2] = k - above; misc[3] = mine; }
+    __syncthreads();
+    tbin = misc[1];
+    need = misc[2];
+    cnt = misc[3];
+    __syncthreads();   // misc[1..2] are reused for the threshold below, wtot for the emission
   }
   if (cnt > NTHR) return block_select_emit(n, k, key, always, emit, fb_hist, fb_wsum, fb_bc);
   for (int i = tid; i < n; i += NTHR) {
@@ -495,27 +492,40 @@ __device__ int block_topk_keyed(int n, int k, KeyFn key, AlwaysFn always, EmitFn
     const uint32_t kv = key(i);
     return kv != 0u && (kv > tkey || (kv == tkey && i <= tidx));
   };
+  // ordered emission: warp w owns items [w * per, (w + 1) * per), per a multiple of 32.  With at most 32
+  // chunks of 32 items per warp, lane c keeps chunk c's ballot from the counting pass for the emitting pass.
   const int per = ((n + NWARPS - 1) / NWARPS + 31) & ~31;
   const int beg = warp * per, end = min(n, beg + per);
+  const bool keep = per <= 1024;
   int mine_n = 0;
-  for (int i0 = beg; i0 < end; i0 += 32) {
+  uint32_t kept = 0u;
+  for (int i0 = beg, c = 0; i0 < end; i0 += 32, ++c) {
     const int i = i0 + lane;
-    mine_n += __popc(__ballot_sync(0xffffffffu, i < end && taken(i)));
+    const uint32_t b = __ballot_sync(0xffffffffu, i < end && taken(i));
+    if (lane == c) kept = b;
+    mine_n += __popc(b);
   }
   if (lane == 0) wtot[warp] = mine_n;
   __syncthreads();
   int before = 0, total = 0;
-  for (int w2 = 0; w2 < NWARPS; ++w2) {
-    const int a = wtot[w2];
-    if (w2 < warp) before += a;
-    total += a;
+  {
+    static_assert(NWARPS <= 32, "one lane per warp total");
+    const int wt = lane < NWARPS ? wtot[lane] : 0;
+    int incl = wt;   // inclusive prefix over warps
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += v;
+    }
+    before = __shfl_sync(0xffffffffu, incl - wt, warp);
+    total = __shfl_sync(0xffffffffu, incl, 31);
   }
   const uint32_t below = (1u << lane) - 1u;
-  for (int i0 = beg; i0 < end; i0 += 32) {
+  for (int i0 = beg, c = 0; i0 < end; i0 += 32, ++c) {
     const int i = i0 + lane;
-    const bool sel = i < end && taken(i);
-    const uint32_t b = __ballot_sync(0xffffffffu, sel);
-    if (sel) emit(before + __popc(b & below), i);
+    const uint32_t b = keep ? __shfl_sync(0xffffffffu, kept, c & 31)
+                            : __ballot_sync(0xffffffffu, i < end && taken(i));
+    if ((b >> lane) & 1u) emit(before + __popc(b & below), i);
     before += __popc(b);
   }
   return total;
