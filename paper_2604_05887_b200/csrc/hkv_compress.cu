@@ -79,9 +79,15 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
         const int jg = j0 + g * 32;
         float gmax = -INFINITY;
         if (all_visible) {
+          float g0 = v[0], g1 = v[1], g2 = v[2], g3 = v[3];   // four short chains instead of one long one
 #pragma unroll
-          for (int c = 0; c < 32; ++c) gmax = fmaxf(gmax, v[c]);
-          gmax *= sc;   // the scale is positive
+          for (int c = 4; c < 32; c += 4) {
+            g0 = fmaxf(g0, v[c]);
+            g1 = fmaxf(g1, v[c + 1]);
+            g2 = fmaxf(g2, v[c + 2]);
+            g3 = fmaxf(g3, v[c + 3]);
+          }
+          gmax = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * sc;   // the scale is positive
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
@@ -91,13 +97,15 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
         }
         if (gmax > -INFINITY) {
           const float m_new = fmaxf(m_run, gmax);
-          float a0 = 0.f, a1 = 0.f;
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
+          for (int c = 0; c < 32; c += 4) {
             a0 += fast_exp2(fmaf(v[c], sc, -m_new));
             a1 += fast_exp2(fmaf(v[c + 1], sc, -m_new));
+            a2 += fast_exp2(fmaf(v[c + 2], sc, -m_new));
+            a3 += fast_exp2(fmaf(v[c + 3], sc, -m_new));
           }
-          z_run = z_run * fast_exp2(m_run - m_new) + (a0 + a1);   // 2^(-inf) = 0 on the first visible group
+          z_run = z_run * fast_exp2(m_run - m_new) + ((a0 + a1) + (a2 + a3));   // 2^(-inf) = 0 on the first visible group
           m_run = m_new;
         }
       });
@@ -126,16 +134,18 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       const int j0 = tile * tc::kKeysPerTile, j = j0 + lane_row;
       const float jf = static_cast<float>(j);
       const bool all_visible = j0 + tc::kKeysPerTile - 1 <= (causal ? C - w : C - 1);   // to every row
-      float acc = 0.f, acc2 = 0.f;
+      float acc = 0.f, acc2 = 0.f, acc3 = 0.f, acc4 = 0.f;
       if (row0 + 128 * half < R) {                     // same for the whole warp
         groups([&](int g, float (&v)[32]) {
           const float4* info = rowinfo + 128 * half + 32 * g;
           if (all_visible) {
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              const float4 r0 = info[c], r1 = info[c + 1];   // a padding row has 1 / sum = 0
+            for (int c = 0; c < 32; c += 4) {
+              const float4 r0 = info[c], r1 = info[c + 1], r2 = info[c + 2], r3 = info[c + 3];   // padding rows: 1 / sum = 0
               acc = fmaf(fast_exp2(fmaf(v[c], sc, -r0.x)), r0.y, acc);
               acc2 = fmaf(fast_exp2(fmaf(v[c + 1], sc, -r1.x)), r1.y, acc2);
+              acc3 = fmaf(fast_exp2(fmaf(v[c + 2], sc, -r2.x)), r2.y, acc3);
+              acc4 = fmaf(fast_exp2(fmaf(v[c + 3], sc, -r3.x)), r3.y, acc4);
             }
           } else {
 #pragma unroll
@@ -147,7 +157,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
           }
         });
       }
-      acc += acc2;
+      acc = (acc + acc2) + (acc3 + acc4);
       // the half-1 warp hands its sums over (two buffers, by tile parity); the half-0 warp adds and
       // stores.  pair_bar is the barrier of this tile's parity: its (n_done / 2)-th use.
       const int slot = (n_done & 1) * 32 + (lane_row & 31);
