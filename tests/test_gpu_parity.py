@@ -99,6 +99,15 @@ def test_causal_window_variant(P):
     P.compare_layer(L, flags=hkv.HKV_OUT_F32 | hkv.HKV_CAUSAL_WINDOW)
 
 
+@pytest.mark.parametrize("w,Hq,Hkv,causal", [(48, 28, 4, False), (48, 28, 4, True), (40, 32, 2, False), (32, 8, 4, True)])
+def test_window_rows_beyond_one_resident_block(P, w, Hq, Hkv, causal):
+    """w * G = 336 and 640 window rows: the window-score kernels run once per block of 256 rows, the later blocks
+    adding to s_w; (32, 8, 4) has 64 rows, a quarter of one block, the rest being padding."""
+    from paper_2604_05887_b200 import binding as hkv
+    L = small(B=2, C=900, cs=16, w=w, Hq=Hq, Hkv=Hkv, budget=0.3, n_steps=1)
+    P.compare_layer(L, flags=hkv.HKV_OUT_F32 | (hkv.HKV_CAUSAL_WINDOW if causal else 0))
+
+
 def test_custom_scale(P):
     L = small(C=300, cs=8)
     P.compare_layer(L, softmax_scale=0.05)
