@@ -143,13 +143,15 @@ def chunk_summaries(k: np.ndarray, cs: int) -> np.ndarray:
     return out
 
 
-def chunk_scores(q: np.ndarray, summaries: np.ndarray) -> np.ndarray:
+def chunk_scores(q: np.ndarray, summaries: np.ndarray, group_max: bool = False) -> np.ndarray:
     """Inner product between the query and each chunk's metadata; for a group of G query heads that
-    share the kv head the score is the sum over the group.  No scale, no softmax: ranking only.
-    float64 -> one rounding to float32.  Returns float32 [n_chunks]."""
+    share the kv head the score is the sum over the group (variant `group_max`: the largest of the
+    group's inner products, i.e. a chunk counts as much as its keenest query head wants it).
+    No scale, no softmax: ranking only.  float64 -> one rounding to float32.  Returns float32 [n_chunks]."""
     Q = bf16_to_f64(q)                                            # [G, d]
     M = bf16_to_f64(summaries)                                    # [n, d]
-    return (M @ Q.T).sum(axis=1).astype(np.float32)
+    dots = M @ Q.T                                                # [n, G]
+    return (dots.max(axis=1) if group_max else dots.sum(axis=1)).astype(np.float32)
 
 
 def n_selected_chunks(budget: int, cs: int, n_chunks: int) -> int:
@@ -262,7 +264,7 @@ def append_token(L, cache: OracleCache, k_new: np.ndarray, v_new: np.ndarray) ->
 
 def decode_layer(L, cache: OracleCache, q: np.ndarray, scale: Optional[float] = None,
                  chunk_override: Optional[Dict[Tuple[int, int], np.ndarray]] = None,
-                 keep_override: Optional[Dict[Tuple[int, int], np.ndarray]] = None):
+                 keep_override: Optional[Dict[Tuple[int, int], np.ndarray]] = None, group_max: bool = False):
     """One decode step of one layer.  q: uint16 [B, Hq, d].
     Static head: attention over its keep-set.  Dynamic head: score the chunks with the query, take
     the top-k, attend over the tokens of those chunks only.  Heads are independent.
@@ -278,7 +280,7 @@ def decode_layer(L, cache: OracleCache, q: np.ndarray, scale: Optional[float] = 
         if hd.kind == 0:
             toks = hd.keep if keep_override is None or (b, h) not in keep_override else np.asarray(keep_override[(b, h)])
         else:
-            s = chunk_scores(qg, hd.summaries)
+            s = chunk_scores(qg, hd.summaries, group_max)
             scores[(b, h)] = s
             sel = select_chunks(s, hd.n_sel)
             if chunk_override is not None and (b, h) in chunk_override:

@@ -330,3 +330,21 @@ def test_selection_exhaustive_subsets_tiny():
     s = sc[(0, 0)].astype(np.float64)
     best = max(itertools.combinations(range(6), 3), key=lambda S: sum(s[list(S)]))
     assert sorted(best) == sel[(0, 0)].tolist()
+
+
+def test_chunk_score_group_max_variant():
+    """The max-over-group variant: hand values, equality with the sum for a group of one, and a case where the two
+    rankings differ (one keen head against many lukewarm ones)."""
+    f = lambda a: hi.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+    m = f([[1, 0], [0, 1], [1, 1]])
+    q = f([[3, 0], [0, 2], [-1, -1]])           # dots: chunk0 (3, 0, -1), chunk1 (0, 2, -1), chunk2 (3, 2, -2)
+    assert o.chunk_scores(q, m, group_max=True).tolist() == [3.0, 2.0, 3.0]
+    assert o.chunk_scores(q, m).tolist() == [2.0, 1.0, 3.0]
+    assert o.chunk_scores(q[:1], m, group_max=True).tolist() == o.chunk_scores(q[:1], m).tolist()
+    q2 = f([[4, 0], [0, 1], [0, 1], [0, 1], [0, 1], [0, 1]])      # chunk0: max 4 / sum 4; chunk1: max 1 / sum 5
+    assert np.argmax(o.chunk_scores(q2, m[:2], group_max=True)) == 0 and np.argmax(o.chunk_scores(q2, m[:2])) == 1
+    rng = np.random.default_rng(3)
+    qq, mm = f(rng.standard_normal((7, 16))), f(rng.standard_normal((9, 16)))
+    ref = [max(float(np.dot(hi.bf16_bits_to_f32(mm[c]).astype(np.float64), hi.bf16_bits_to_f32(qq[g]).astype(np.float64)))
+               for g in range(7)) for c in range(9)]
+    assert np.allclose(o.chunk_scores(qq, mm, group_max=True), np.float32(ref), rtol=0, atol=0)
