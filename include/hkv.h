@@ -52,6 +52,10 @@ typedef enum {
 #define HKV_CAUSAL_WINDOW 1u /* mask key j > position of the window row inside S_w (variant; the
                                 paper's equation has no mask)                                  */
 #define HKV_OUT_F32 2u       /* hkv_decode_attn writes float32 instead of bf16                 */
+#define HKV_GROUP_MAX 4u     /* chunk score of a GQA group = the largest of its query heads' inner
+                                products with the chunk mean instead of their sum (variant: the
+                                paper scores per head and does not say how a shared KV head
+                                combines its group)                                            */
 
 /* Geometry of one layer's cache.  Supported: head_dim = 128, 1 <= n_q_heads / n_kv_heads <= 16,
  * chunk_size >= 1, 1 <= obs_window <= every seq_len. */

@@ -18,6 +18,7 @@ _LIB_PATH = os.environ.get("HKV_LIB") or os.path.join(os.path.dirname(os.path.ab
 HKV_OK = 0
 HKV_CAUSAL_WINDOW = 1
 HKV_OUT_F32 = 2
+HKV_GROUP_MAX = 4
 
 STATUS_NAMES = {0: "HKV_OK", 1: "HKV_ERR_INVALID_ARG", 2: "HKV_ERR_SHAPE", 3: "HKV_ERR_BUDGET",
                 4: "HKV_ERR_WORKSPACE", 5: "HKV_ERR_UNSUPPORTED", 6: "HKV_ERR_CUDA", 7: "HKV_ERR_TIMEOUT",

@@ -23,7 +23,7 @@ hkv_status check_config(const hkv_config* cfg) {
   if (cfg->head_dim != kHeadDim) return HKV_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) return HKV_ERR_UNSUPPORTED;
   if (cfg->chunk_size < 1 || cfg->obs_window < 1) return HKV_ERR_SHAPE;
-  if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32)) return HKV_ERR_INVALID_ARG;
+  if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32 | HKV_GROUP_MAX)) return HKV_ERR_INVALID_ARG;
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return HKV_ERR_INVALID_ARG;
   if (static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads > 60000) return HKV_ERR_UNSUPPORTED;
   if (cfg->append_capacity < 0 || cfg->append_capacity > (1 << 24)) return HKV_ERR_SHAPE;
@@ -248,7 +248,7 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
     const Header& H = c->hdr;
     const Header& H0 = caches[0]->hdr;
     if (H.group != H0.group || H.n_q_heads != H0.n_q_heads || H.n_kv_heads != H0.n_kv_heads ||
-        H.chunk_size != H0.chunk_size || H.scale != H0.scale || ((H.flags ^ H0.flags) & HKV_OUT_F32))
+        H.chunk_size != H0.chunk_size || H.scale != H0.scale || ((H.flags ^ H0.flags) & (HKV_OUT_F32 | HKV_GROUP_MAX)))
       return HKV_ERR_SHAPE;
     P.cache[i] = c->dev_base;
     P.q[i] = q[i];
@@ -265,6 +265,7 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   P.scale_log2e = H0.scale * 1.4426950408889634f;
   P.phase = (do_select ? kPhaseSelect : 0u) | (do_attend ? kPhaseAttend : 0u);
   P.out_f32 = (H0.flags & HKV_OUT_F32) ? 1u : 0u;
+  P.group_max = (H0.flags & HKV_GROUP_MAX) ? 1u : 0u;
   const int* max_active = nullptr;
   if (decode_cluster_caps(P.group, &max_active) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
   const int total_units = P.unit_prefix[n];
@@ -341,7 +342,7 @@ hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void*
     if (!caches[i]) return HKV_ERR_INVALID_ARG;
     const hkv_config &a = caches[i]->cfg, &b = caches[0]->cfg;
     if (a.batch != b.batch || a.n_q_heads != b.n_q_heads || a.head_dim != b.head_dim ||
-        ((a.flags ^ b.flags) & HKV_OUT_F32))
+        ((a.flags ^ b.flags) & (HKV_OUT_F32 | HKV_GROUP_MAX)))
       return HKV_ERR_SHAPE;
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -395,17 +395,39 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[kk & 1][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
         }
-        // chunk score = sum over the group's heads of <q_g, mean_c>
-        float v0 = 0.f, v1 = 0.f;
+        // chunk score = sum over the group's heads of <q_g, mean_c> (variant: their maximum; the
+        // columns past the group hold zero queries and must not take part in it)
+        float v0, v1;
+        if (P.group_max) {
+          v0 = v1 = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          v0 += (acc[0][nt][0] + acc[1][nt][0]) + (acc[0][nt][1] + acc[1][nt][1]);
-          v1 += (acc[0][nt][2] + acc[1][nt][2]) + (acc[0][nt][3] + acc[1][nt][3]);
+          for (int nt = 0; nt < NT; ++nt) {
+            const int h0 = nt * 8 + 2 * t;
+            if (h0 < G) {
+              v0 = fmaxf(v0, acc[0][nt][0] + acc[1][nt][0]);
+              v1 = fmaxf(v1, acc[0][nt][2] + acc[1][nt][2]);
+            }
+            if (h0 + 1 < G) {
+              v0 = fmaxf(v0, acc[0][nt][1] + acc[1][nt][1]);
+              v1 = fmaxf(v1, acc[0][nt][3] + acc[1][nt][3]);
+            }
+          }
+          v0 = fmaxf(v0, __shfl_xor_sync(0xffffffffu, v0, 1));
+          v0 = fmaxf(v0, __shfl_xor_sync(0xffffffffu, v0, 2));
+          v1 = fmaxf(v1, __shfl_xor_sync(0xffffffffu, v1, 1));
+          v1 = fmaxf(v1, __shfl_xor_sync(0xffffffffu, v1, 2));
+        } else {
+          v0 = v1 = 0.f;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            v0 += (acc[0][nt][0] + acc[1][nt][0]) + (acc[0][nt][1] + acc[1][nt][1]);
+            v1 += (acc[0][nt][2] + acc[1][nt][2]) + (acc[0][nt][3] + acc[1][nt][3]);
+          }
+          v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+          v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
+          v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+          v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
         }
-        v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
-        v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
-        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-        v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
         const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
         if (!fast) {   // too many chunks for shared memory: the selection reads the scores from global memory
           if (t == 0 && c0 < n_chunks) gscores[c0] = v0;

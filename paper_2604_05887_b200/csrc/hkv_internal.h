@@ -73,6 +73,7 @@ struct DecodeParams {
   uint32_t phase;      // kPhaseSelect | kPhaseAttend
   uint32_t out_f32;
   uint32_t pdl;        // launched with programmatic stream serialization
+  uint32_t group_max;  // chunk score = max over the group's heads instead of their sum
   int32_t unit_prefix[kMaxMulti + 1];
   char* cache[kMaxMulti];
   const void* q[kMaxMulti];

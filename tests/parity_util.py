@@ -48,6 +48,7 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
                   softmax_scale=0.0):
     """Compress + decode one layer on the GPU and on the oracle; assert parity. Returns a report."""
     causal = bool(flags & hkv.HKV_CAUSAL_WINDOW)
+    group_max = bool(flags & hkv.HKV_GROUP_MAX)
     lc = LayerCache(L, flags=flags, token_scores=token_scores, keep_workspace=True, softmax_scale=softmax_scale)
     code, detail = hkv.hkv_last_device_error(lc.handle)
     assert code == 0, f"device error {code}/{detail} after compress"
@@ -84,7 +85,7 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
         torch.cuda.synchronize()
         code, detail = hkv.hkv_last_device_error(lc.handle)
         assert code == 0, f"device error {code}/{detail} after decode"
-        _, ref_sel, ref_scores = o.decode_layer(L, oc, q_bits, scale=softmax_scale or None)
+        _, ref_sel, ref_scores = o.decode_layer(L, oc, q_bits, scale=softmax_scale or None, group_max=group_max)
         chunk_override = {}
         for (b, h) in units:
             hd = oc.heads[(b, h)]
@@ -101,7 +102,8 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
             if n:
                 chunk_override[(b, h)] = gsel
         ref_out, _, _ = o.decode_layer(L, oc, q_bits, chunk_override=chunk_override or None,
-                                       keep_override=keep_override or None, scale=softmax_scale or None)
+                                       keep_override=keep_override or None, scale=softmax_scale or None,
+                                       group_max=group_max)
         G = L.group
         rows = np.concatenate([np.arange(h * G, (h + 1) * G) + 0 for (_, h) in units]) if units else []
         g_out = out.float().cpu().numpy()

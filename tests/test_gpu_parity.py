@@ -108,6 +108,22 @@ def test_window_rows_beyond_one_resident_block(P, w, Hq, Hkv, causal):
     P.compare_layer(L, flags=hkv.HKV_OUT_F32 | (hkv.HKV_CAUSAL_WINDOW if causal else 0))
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(28, 4), (32, 2), (4, 4), (16, 2)])
+def test_group_max_scoring_variant(P, Hq, Hkv):
+    """HKV_GROUP_MAX: the chunk score is the largest inner product of the group (groups of 7, 16, 1, 8)."""
+    from paper_2604_05887_b200 import binding as hkv
+    L = small(B=2, C=1100, cs=16, w=8, Hq=Hq, Hkv=Hkv, budget=0.25, n_steps=2, head_type=np.ones((2, Hkv), np.uint8))
+    rep = P.compare_layer(L, flags=hkv.HKV_OUT_F32 | hkv.HKV_GROUP_MAX)
+    assert rep["stats"]["n_dynamic"] == 2 * Hkv
+
+
+def test_second_geometry_qwen25_vl_3b(P):
+    """16 query / 2 KV heads (group of 8), head_dim 128: the smaller model the paper also evaluates."""
+    L = small(B=3, C=5000, cs=32, w=32, Hq=16, Hkv=2, budget=0.1, n_steps=2)
+    rep = P.compare_layer(L)
+    assert rep["stats"]["n_static"] + rep["stats"]["n_dynamic"] == 6
+
+
 def test_custom_scale(P):
     L = small(C=300, cs=8)
     P.compare_layer(L, softmax_scale=0.05)
