@@ -166,6 +166,39 @@ def layer_algo_bytes(L) -> int:
     return tot
 
 
+def measure_classification(L, dev, n_text: int = 256):
+    """hkv_classify_heads on one layer's keys with `n_text` text-token queries per sequence (the step before the
+    budgets and the compression; not part of the decode metric)."""
+    import torch
+    import hkv_inputs as hi
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import to_device_bf16
+    q_text, counts = hi.text_queries(L, n_text, ragged=False)
+    cfg = hkv.hkv_config(batch=L.batch, n_q_heads=L.n_q_heads, n_kv_heads=L.n_kv_heads, head_dim=L.head_dim,
+                         max_seq_len=L.max_seq_len, chunk_size=L.chunk_size, obs_window=L.obs_window,
+                         softmax_scale=0.0, flags=0, append_capacity=0)
+    _, ws_bytes = hkv.hkv_classify_workspace(cfg, n_text)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    scores = torch.zeros((L.batch, L.n_kv_heads), dtype=torch.float64, device=dev)
+    types = torch.zeros((L.batch, L.n_kv_heads), dtype=torch.uint8, device=dev)
+    k, q = to_device_bf16(L.k, dev), to_device_bf16(q_text, dev)
+    times = []
+    for _ in range(4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        hkv.hkv_classify_heads(cfg, k, q, L.seq_lens, counts, 0.05, 0.9, ws, scores, types)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    rows = int(sum(int(c) for c in counts)) * L.n_q_heads
+    cols = float(sum(int(c) * int(t) for c, t in zip(L.seq_lens, counts))) * L.n_q_heads   # softmax entries
+    ms = min(times[1:])
+    return {"what": "hkv_classify_heads, layer 0: text-centric attention rows -> top-5% sums -> score -> label",
+            "text_tokens_per_sequence": n_text, "rows": rows, "ms": ms, "us_per_row": ms * 1e3 / rows,
+            "logit_TFLOPs": cols * 2 * L.head_dim / (ms * 1e-3) / 1e12,
+            "static_heads_at_theta_0.9": int((types == 0).sum().item()), "heads": L.batch * L.n_kv_heads}
+
+
 def measure_other_workload(workload: str, n_caches: int, seed: int, dev, peak: float):
     """Per-launch time of the decode kernel on another workload: `n_caches` independent one-layer
     caches (distinct seeds, together larger than L2) replayed round-robin from one CUDA graph."""
@@ -529,6 +562,7 @@ def main():
         del caches, qs, outs
         torch.cuda.empty_cache()
         line["other_workloads"] = [measure_other_workload("cfg4", 4, args.seed + 4, dev, peak)]
+        line["next_rows"] = [measure_classification(L0, dev)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt, n = oracle_decode_timing(L0, args.cpu_seconds)
         b0 = stats[0]["algorithmic_bytes_per_step"]
