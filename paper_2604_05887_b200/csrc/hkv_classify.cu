@@ -280,6 +280,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
       return fminf(q, 1.f);          // every bit pattern stays in [0, bits(1)]
     };
     float z = 0.f;
+#pragma unroll 4
     for (int i = tid; i < n4; i += kClsRowThreads) {
       const float4 v = row4[i];
       const float4 q = make_float4(prob(v.x), prob(v.y), prob(v.z), prob(v.w));
@@ -298,6 +299,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
     float top = 0.f;
     for (;;) {
       if (need == cnt) {                      // the whole bin is inside the top k
+#pragma unroll 4
         for (int i = tid; i < n4; i += kClsRowThreads) {
           const float4 q = row4[i];
           top += (((__float_as_uint(q.x) >> shift) >= prefix ? q.x : 0.f) +
@@ -311,6 +313,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
         // sum what lies above the bin, collect the bin's entries (a warp that meets some reserves
         // their slots with one atomic) and sort them exactly (descending; equal values in an
         // arbitrary but complete order): the first `need` join the sum
+#pragma unroll 4
         for (int i0 = warp * 32; i0 < n4; i0 += kClsRowThreads) {
           const int i = i0 + lane;
           const float4 q = i < n4 ? row4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
