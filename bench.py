@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0           # the denominator the task statement names ("
 N_LAYERS = {"cfg0": 1, "cfg1": 28, "cfg2": 28, "cfg3": 28, "cfg4": 1}
 # DRAM bytes per launch of the flash-decode kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 26.81e6}   # profiles/decode_kernel_cfg2.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 26.85e6}   # profiles/decode_kernel_cfg2.md
 
 
 def layer_inputs(workload: str, layer: int, seed: int, threads: int):
