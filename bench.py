@@ -550,7 +550,7 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
         "e2e": {"value": world_bytes / t_e2e / 1e9, "unit": "GB/s", "us_per_step": t_e2e * 1e6,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "how": "hkv_decode_step_host: pinned host queries of all layers -> device, one decode launch per layer, outputs -> pinned host, copies enqueued by the C-ABI call, all inside the timed graph (the per-layer host entry point hkv_decode_attn_host costs two PCIe round trips per layer: 990 us/step)"},
+                "how": "hkv_decode_step_host: pinned host queries of all layers -> device (first layer's ahead, the rest beside the first layers), one decode launch per layer, outputs -> pinned host in four groups beside the later layers, copies enqueued by the C-ABI call, all inside the timed graph (the per-layer host entry point hkv_decode_attn_host costs two PCIe round trips per layer: 990 us/step)"},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk.summary(),
         "device_error": [code, detail],

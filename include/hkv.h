@@ -182,9 +182,14 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
 hkv_status hkv_append(hkv_cache* cache, const void* k_new, const void* v_new, void* stream);
 
 /* One decode step of a whole model with HOST buffers (Appendix A's per-step procedure, layer after
- * layer): the queries of all n layers are copied to the device in one transfer, one hkv_decode_attn
- * launch per layer follows (caches[i] with layer i's slice, in order), and all outputs return in
- * one transfer — everything enqueued on `stream`.
+ * layer): the queries of the first layer are copied to the device on `stream`, those of the other
+ * layers meanwhile on a second stream the library keeps per device; one hkv_decode_attn launch per
+ * layer follows on `stream` (caches[i] with layer i's slice, in order); the outputs return in four
+ * groups of layers, the first three beside the layers still running, the last on `stream`, which
+ * also waits for the second stream before the call's work counts as finished.  From the caller's
+ * side everything is ordered on `stream`; the call may be captured in a CUDA graph (the second
+ * stream forks from and joins `stream` by events).  The first call on a device creates that stream
+ * and its events.
  *   q_host, out_host  host [n, B, Hq, d] (pinned for truly asynchronous copies); bf16 / float32 as for hkv_decode_attn
  *   q_dev, out_dev    caller-owned device staging buffers of the same sizes
  * All caches must share one geometry (batch, heads, output type). */

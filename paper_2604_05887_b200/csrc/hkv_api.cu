@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -335,6 +336,39 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
   return HKV_OK;
 }
 
+namespace {
+// A second stream and a few events per device for hkv_decode_step_host: the queries of the layers
+// after the first travel to the device while the first layer runs, and the outputs of all but the
+// last group of layers travel back while later layers run.  Created on first use, never destroyed.
+constexpr int kStepGroups = 4;
+struct StepSide {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, q_done = nullptr, q_done2 = nullptr, join = nullptr, out[kStepGroups] = {};
+  bool ready = false;
+};
+StepSide g_step_side[64];
+std::mutex g_step_mutex;
+
+StepSide* step_side() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_step_mutex);
+  StepSide& s = g_step_side[dev];
+  if (!s.ready) {
+    bool ok = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.q_done, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.q_done2, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kStepGroups; ++i)
+      ok = cudaEventCreateWithFlags(&s.out[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return nullptr; }
+    s.ready = true;
+  }
+  return &s;
+}
+}  // namespace
+
 hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void* q_host, void* out_host, void* q_dev,
                                 void* out_dev, void* stream) {
   if (!caches || n < 1 || !q_host || !out_host || !q_dev || !out_dev) return HKV_ERR_INVALID_ARG;
@@ -348,13 +382,55 @@ hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void*
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t per = static_cast<size_t>(caches[0]->cfg.batch) * caches[0]->cfg.n_q_heads * caches[0]->cfg.head_dim;
   const size_t out_elt = (caches[0]->hdr.flags & HKV_OUT_F32) ? 4 : 2;
-  if (cudaMemcpyAsync(q_dev, q_host, per * 2 * n, cudaMemcpyHostToDevice, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
-  for (int i = 0; i < n; ++i) {
-    hkv_status st = hkv_decode_attn(caches[i], static_cast<const char*>(q_dev) + per * 2 * i,
-                                    static_cast<char*>(out_dev) + per * out_elt * i, stream);
-    if (st != HKV_OK) return st;
+  const char* qh = static_cast<const char*>(q_host);
+  char* qd = static_cast<char*>(q_dev);
+  char* oh = static_cast<char*>(out_host);
+  char* od = static_cast<char*>(out_dev);
+  StepSide* side = n >= 2 ? step_side() : nullptr;
+  const int q_split = std::min(n, 4);   // layers 1 .. q_split - 1 get their queries in a first, short transfer
+  bool ok = true;
+  auto cu = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
+
+  // queries: the first layer's on the caller's stream, the rest beside it
+  cu(cudaMemcpyAsync(qd, qh, per * 2 * (side ? 1 : n), cudaMemcpyHostToDevice, s));
+  if (side) {
+    cu(cudaEventRecord(side->fork, s));
+    cu(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    // a short piece first, so that the second layer is not held up by the whole transfer
+    cu(cudaMemcpyAsync(qd + per * 2, qh + per * 2, per * 2 * (q_split - 1), cudaMemcpyHostToDevice, side->stream));
+    cu(cudaEventRecord(side->q_done, side->stream));
+    if (q_split < n) {
+      cu(cudaMemcpyAsync(qd + per * 2 * q_split, qh + per * 2 * q_split, per * 2 * (n - q_split), cudaMemcpyHostToDevice,
+                         side->stream));
+      cu(cudaEventRecord(side->q_done2, side->stream));
+    }
   }
-  if (cudaMemcpyAsync(out_host, out_dev, per * out_elt * n, cudaMemcpyDeviceToHost, s) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  if (!ok) { cudaGetLastError(); return HKV_ERR_CUDA; }
+  // layers in order; after each group of layers but the last, its outputs start their way back
+  const int groups = side ? std::min(kStepGroups, n) : 1;
+  int done_out = 0;   // layers whose outputs have been sent
+  for (int i = 0; i < n; ++i) {
+    if (side && i == 1) cu(cudaStreamWaitEvent(s, side->q_done, 0));
+    if (side && i == q_split && q_split < n) cu(cudaStreamWaitEvent(s, side->q_done2, 0));
+    hkv_status st = hkv_decode_attn(caches[i], qd + per * 2 * i, od + per * out_elt * i, stream);
+    if (st != HKV_OK) return st;
+    const int g = static_cast<int>((static_cast<long long>(i + 1) * groups) / n);   // groups complete after layer i
+    const int g_prev = static_cast<int>((static_cast<long long>(i) * groups) / n);
+    if (side && g > g_prev && g < groups) {
+      cu(cudaEventRecord(side->out[g - 1], s));
+      cu(cudaStreamWaitEvent(side->stream, side->out[g - 1], 0));
+      cu(cudaMemcpyAsync(oh + per * out_elt * done_out, od + per * out_elt * done_out,
+                         per * out_elt * (i + 1 - done_out), cudaMemcpyDeviceToHost, side->stream));
+      done_out = i + 1;
+    }
+  }
+  cu(cudaMemcpyAsync(oh + per * out_elt * done_out, od + per * out_elt * done_out, per * out_elt * (n - done_out),
+                     cudaMemcpyDeviceToHost, s));
+  if (side) {   // the caller's stream ends the step only when the side copies have ended
+    cu(cudaEventRecord(side->join, side->stream));
+    cu(cudaStreamWaitEvent(s, side->join, 0));
+  }
+  if (!ok) { cudaGetLastError(); return HKV_ERR_CUDA; }
   return HKV_OK;
 }
 
