@@ -88,3 +88,25 @@ def test_split_plan_is_one_wave_for_bench_shape(hkv):
     cfg = _cfg(hkv, batch=4, max_seq_len=32768, chunk_size=64)
     cache_bytes, _ = hkv.hkv_plan(cfg, sl, ht, bu)
     assert cache_bytes < 2 * 256 * 32768 * 16      # far below the full KV of the layer
+
+
+def test_classification_workspace_sizes(hkv):
+    """hkv_classify_workspace is host arithmetic: 256 B error word + row sums + at least 16 rows of logits per
+    (sequence, kv head) for the minimum, every row (up to half a gigabyte of logits) for the preferred size."""
+    cfg = _cfg(hkv, max_seq_len=1000)
+    lo, hi = hkv.hkv_classify_workspace(cfg, 10)
+    units, r_max, c_stride = 2 * 4, 10 * 7, 1024          # rows padded to a multiple of 128 floats
+    head = 256 + -(-units * r_max * 4 // 256) * 256
+    assert lo == head + 16 * c_stride * 4 * units
+    assert hi == head + 80 * c_stride * 4 * units          # 70 rows rounded up to a multiple of 16
+    lo2, hi2 = hkv.hkv_classify_workspace(cfg, 1000)
+    assert lo2 > lo and hi2 > hi and lo2 <= hi2
+    big = _cfg(hkv, batch=16, max_seq_len=32768)
+    lo3, hi3 = hkv.hkv_classify_workspace(big, 768)
+    assert hi3 - lo3 < (512 << 20) + (16 << 20) and hi3 > (256 << 20)
+    for bad, status in ((dict(head_dim=64), 5), (dict(n_q_heads=30), 2), (dict(batch=0), 2)):
+        with pytest.raises(hkv.HkvError) as e:
+            hkv.hkv_classify_workspace(_cfg(hkv, **bad), 10)
+        assert e.value.status == status
+    with pytest.raises(hkv.HkvError):
+        hkv.hkv_classify_workspace(cfg, 0)
