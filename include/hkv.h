@@ -16,8 +16,10 @@
  * "Head" always means KV head; the G = n_q_heads / n_kv_heads query heads of a group share it.
  *
  * Conventions
- *   - plain C linkage; no exception crosses the boundary; no global state; every call returns a
- *     status.  Argument errors are found on the host before anything is launched.
+ *   - plain C linkage; no exception crosses the boundary; every call returns a status.  Argument
+ *     errors are found on the host before anything is launched.  Global state is limited to what
+ *     two entry points document: the helper stream of hkv_decode_step_host and the fixed scratch of
+ *     hkv_topk_chunks_noalloc.
  *   - "dev" pointers are device (HBM) addresses on the current CUDA device, "host" pointers are
  *     ordinary host memory.  bf16 tensors are passed as void*.
  *   - the caller owns every device buffer, including cache_mem and workspace.  The library never
@@ -121,6 +123,9 @@ hkv_status hkv_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_
  * Dynamic head: chunk mean = float32 sum of the chunk's keys in token order / chunk length, rounded
  * to nearest-even bf16; the last chunk may be shorter.
  * k, v, q_obs, token_scores and is_text may be released once the stream has passed this call.
+ * The window-score kernels (and hkv_classify_heads) run on the tcgen05 tensor cores: while they run,
+ * each of their thread blocks holds all tensor memory and nearly all shared memory of its SM, so
+ * kernels of other streams that need tensor memory wait for them.
  * On success *out receives a handle to free with hkv_cache_destroy. */
 hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
                         const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
