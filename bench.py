@@ -199,6 +199,41 @@ def measure_classification(L, dev, n_text: int = 256):
             "static_heads_at_theta_0.9": int((types == 0).sum().item()), "heads": L.batch * L.n_kv_heads}
 
 
+def measure_offload(L, dev, launches: int = 10):
+    """One layer with HKV_OFFLOAD_DYNAMIC (the paper's placement: dynamic heads' K/V in pinned host memory, the
+    selected chunks cross PCIe inside the decode kernel): time per launch from a CUDA graph of `launches`."""
+    import torch
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    lc = LayerCache(L, flags=hkv.HKV_OFFLOAD_DYNAMIC, device=dev)
+    q, out = to_device_bf16(L.q[0], dev), lc.new_out()
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            hkv.hkv_decode_attn(lc.handle, q, out)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(launches):
+                hkv.hkv_decode_attn(lc.handle, q, out)
+        times = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3 / launches)
+    us = min(times[1:])
+    host_bytes = sum(512 * min(int(L.seq_lens[b]), -(-int(L.budgets[b, h]) // L.chunk_size) * L.chunk_size)
+                     for b in range(L.batch) for h in range(L.n_kv_heads) if L.head_type[b, h] == 1)
+    code, detail = hkv.hkv_last_device_error(lc.handle)
+    lc.close()
+    return {"what": "HKV_OFFLOAD_DYNAMIC, layer 0: dynamic heads' K/V in pinned host memory, selected chunks read over PCIe by the decode kernel",
+            "us_per_launch": us, "host_bytes_per_launch": host_bytes, "pcie_GBps": host_bytes / us / 1e3,
+            "device_error": [code, detail]}
+
+
 def measure_other_workload(workload: str, n_caches: int, seed: int, dev, peak: float):
     """Per-launch time of the decode kernel on another workload: `n_caches` independent one-layer
     caches (distinct seeds, together larger than L2) replayed round-robin from one CUDA graph."""
@@ -562,7 +597,7 @@ def main():
         del caches, qs, outs
         torch.cuda.empty_cache()
         line["other_workloads"] = [measure_other_workload("cfg4", 4, args.seed + 4, dev, peak)]
-        line["next_rows"] = [measure_classification(L0, dev)]
+        line["next_rows"] = [measure_classification(L0, dev), measure_offload(L0, dev)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt, n = oracle_decode_timing(L0, args.cpu_seconds)
         b0 = stats[0]["algorithmic_bytes_per_step"]

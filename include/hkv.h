@@ -59,6 +59,11 @@ typedef enum {
                                 paper scores per head and does not say how a shared KV head
                                 combines its group)                                            */
 
+#define HKV_OFFLOAD_DYNAMIC 8u /* the K/V planes of the dynamic heads live in pinned host memory and
+                                the selected chunks cross PCIe every step (the paper's own
+                                placement, Section 3.3 / Appendix A); only with hkv_plan_offload /
+                                hkv_compress_offload                                           */
+
 /* Geometry of one layer's cache.  Supported: head_dim = 128, 1 <= n_q_heads / n_kv_heads <= 16,
  * chunk_size >= 1, 1 <= obs_window <= every seq_len. */
 typedef struct {
@@ -132,6 +137,28 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
                         const uint8_t* head_type, const int32_t* budgets, void* cache_mem,
                         size_t cache_bytes, void* workspace, size_t workspace_bytes, void* stream,
                         hkv_cache** out);
+
+/* The paper's placement of the dynamic heads' KV (Section 3.3: dynamic-head KV is offloaded to CPU
+ * memory and the chunks a step selects are fetched to the GPU; Appendix A).  Same as hkv_plan /
+ * hkv_compress with cfg->flags carrying HKV_OFFLOAD_DYNAMIC, except that the K and V planes of the
+ * dynamic heads are written to `host_mem` instead of cache_mem (chunk means, scores and index lists
+ * stay on the device).
+ *   host_mem   pinned host memory the device can address at the same pointer value (cudaHostAlloc /
+ *              cudaMallocHost / a registered range under unified addressing), >= host_bytes, 256-B
+ *              aligned, owned by the caller, alive as long as the handle is used
+ * Every later call on the handle (decode, append, getters) works unchanged: the decode kernel's bulk
+ * copies read the selected chunks straight from host memory, so a step moves them over PCIe and no
+ * staging buffer or extra launch exists.  Without dynamic heads host_bytes is 0 and host_mem may be
+ * NULL.  The plain hkv_plan / hkv_compress reject the flag (HKV_ERR_INVALID_ARG), and these two
+ * reject its absence. */
+hkv_status hkv_plan_offload(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type,
+                            const int32_t* budgets, size_t* cache_bytes, size_t* workspace_bytes,
+                            size_t* host_bytes);
+hkv_status hkv_compress_offload(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                                const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                                const uint8_t* head_type, const int32_t* budgets, void* cache_mem,
+                                size_t cache_bytes, void* host_mem, size_t host_bytes, void* workspace,
+                                size_t workspace_bytes, void* stream, hkv_cache** out);
 
 /* One decode step over the compressed cache (Appendix A: score chunks by the inner product of the
  * query with the chunk metadata, take the top chunks, attend together with the static cache).

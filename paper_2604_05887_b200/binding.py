@@ -19,6 +19,7 @@ HKV_OK = 0
 HKV_CAUSAL_WINDOW = 1
 HKV_OUT_F32 = 2
 HKV_GROUP_MAX = 4
+HKV_OFFLOAD_DYNAMIC = 8
 
 STATUS_NAMES = {0: "HKV_OK", 1: "HKV_ERR_INVALID_ARG", 2: "HKV_ERR_SHAPE", 3: "HKV_ERR_BUDGET",
                 4: "HKV_ERR_WORKSPACE", 5: "HKV_ERR_UNSUPPORTED", 6: "HKV_ERR_CUDA", 7: "HKV_ERR_TIMEOUT",
@@ -29,7 +30,7 @@ EXPORTS = ["hkv_plan", "hkv_compress", "hkv_decode_attn", "hkv_decode_attn_multi
            "hkv_get_static_indices", "hkv_get_selected_chunks", "hkv_get_chunk_scores", "hkv_get_summaries",
            "hkv_window_scores_offset", "hkv_cache_stats", "hkv_last_device_error", "hkv_status_string",
            "hkv_topk_chunks_noalloc", "hkv_decode_cluster_capacity", "hkv_allocate_budgets", "hkv_append", "hkv_decode_step_host",
-           "hkv_classify_workspace", "hkv_classify_heads"]
+           "hkv_classify_workspace", "hkv_classify_heads", "hkv_plan_offload", "hkv_compress_offload"]
 
 
 class hkv_config(C.Structure):
@@ -66,6 +67,10 @@ def _load() -> C.CDLL:
     lib.hkv_plan.argtypes = [cfgp, i32p, u8p, i32p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.hkv_compress.argtypes = [cfgp, vp, vp, vp, vp, vp, i32p, u8p, i32p, vp, C.c_size_t, vp, C.c_size_t, vp,
                                  C.POINTER(vp)]
+    lib.hkv_plan_offload.argtypes = [cfgp, i32p, u8p, i32p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t),
+                                     C.POINTER(C.c_size_t)]
+    lib.hkv_compress_offload.argtypes = [cfgp, vp, vp, vp, vp, vp, i32p, u8p, i32p, vp, C.c_size_t, vp, C.c_size_t,
+                                         vp, C.c_size_t, vp, C.POINTER(vp)]
     lib.hkv_decode_attn.argtypes = [vp, vp, vp, vp]
     lib.hkv_decode_attn_multi.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int32, vp]
     lib.hkv_select_chunks.argtypes = [vp, vp, vp]
@@ -165,6 +170,33 @@ def hkv_compress(cfg: hkv_config, k, v, q_obs, token_scores, is_text, seq_lens, 
                             _dev(cache_mem), cache_mem.numel() * cache_mem.element_size(),
                             _dev(workspace), workspace.numel() * workspace.element_size(),
                             _stream(stream), C.byref(handle)), "hkv_compress")
+    return handle.value
+
+
+def hkv_plan_offload(cfg: hkv_config, seq_lens, head_type, budgets):
+    """-> (cache_bytes, workspace_bytes, host_bytes) for the variant with the dynamic heads' K/V in host memory."""
+    sl, ht, bu = _i32(seq_lens), _u8(head_type), _i32(budgets)
+    cb, wb, hb = C.c_size_t(0), C.c_size_t(0), C.c_size_t(0)
+    _check(lib.hkv_plan_offload(C.byref(cfg), _ptr(sl, C.c_int32), _ptr(ht, C.c_uint8), _ptr(bu, C.c_int32),
+                                C.byref(cb), C.byref(wb), C.byref(hb)), "hkv_plan_offload")
+    return int(cb.value), int(wb.value), int(hb.value)
+
+
+def hkv_compress_offload(cfg: hkv_config, k, v, q_obs, token_scores, is_text, seq_lens, head_type, budgets,
+                         cache_mem, host_mem, workspace, stream=None) -> int:
+    """hkv_compress with the dynamic heads' K/V planes written to `host_mem`, a pinned CPU tensor (or None when
+    the layer has no dynamic head)."""
+    sl, ht, bu = _i32(seq_lens), _u8(head_type), _i32(budgets)
+    handle = C.c_void_p(None)
+    if host_mem is not None and (host_mem.is_cuda or not host_mem.is_pinned() or not host_mem.is_contiguous()):
+        raise ValueError("expected a contiguous pinned CPU tensor")
+    hp = host_mem.data_ptr() if host_mem is not None else None
+    hn = host_mem.numel() * host_mem.element_size() if host_mem is not None else 0
+    _check(lib.hkv_compress_offload(C.byref(cfg), _dev(k), _dev(v), _dev(q_obs), _dev(token_scores), _dev(is_text),
+                                    _ptr(sl, C.c_int32), _ptr(ht, C.c_uint8), _ptr(bu, C.c_int32),
+                                    _dev(cache_mem), cache_mem.numel() * cache_mem.element_size(), hp, hn,
+                                    _dev(workspace), workspace.numel() * workspace.element_size(),
+                                    _stream(stream), C.byref(handle)), "hkv_compress_offload")
     return handle.value
 
 

@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <initializer_list>
 #include <mutex>
 #include <cstring>
 #include <new>
@@ -24,7 +25,7 @@ hkv_status check_config(const hkv_config* cfg) {
   if (cfg->head_dim != kHeadDim) return HKV_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) return HKV_ERR_UNSUPPORTED;
   if (cfg->chunk_size < 1 || cfg->obs_window < 1) return HKV_ERR_SHAPE;
-  if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32 | HKV_GROUP_MAX)) return HKV_ERR_INVALID_ARG;
+  if (cfg->flags & ~(HKV_CAUSAL_WINDOW | HKV_OUT_F32 | HKV_GROUP_MAX | HKV_OFFLOAD_DYNAMIC)) return HKV_ERR_INVALID_ARG;
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return HKV_ERR_INVALID_ARG;
   if (static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads > 60000) return HKV_ERR_UNSUPPORTED;
   if (cfg->append_capacity < 0 || cfg->append_capacity > (1 << 24)) return HKV_ERR_SHAPE;
@@ -33,9 +34,11 @@ hkv_status check_config(const hkv_config* cfg) {
 
 // Fills every host-side field of `c` (units, splits, header with offsets, sizes).
 hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type, const int32_t* budgets,
-                      hkv_cache& c, int64_t* ws_rowstat_off, int* n_col_tiles_max) {
+                      hkv_cache& c, int64_t* ws_rowstat_off, int* n_col_tiles_max, bool offload = false) {
   hkv_status st = check_config(cfg);
   if (st != HKV_OK) return st;
+  // the flag and the entry point go together: the dynamic planes need a second buffer
+  if (((cfg->flags & HKV_OFFLOAD_DYNAMIC) != 0) != offload) return HKV_ERR_INVALID_ARG;
   if (!seq_lens || !head_type || !budgets) return HKV_ERR_INVALID_ARG;
   const int B = cfg->batch, Hkv = cfg->n_kv_heads, G = cfg->n_q_heads / Hkv, cs = cfg->chunk_size, w = cfg->obs_window;
   for (int b = 0; b < B; ++b) {
@@ -116,11 +119,16 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
       u.tail_sum_off = off;  off = align_up(off + 4ll * kHeadDim);
     }
   }
+  // K and V planes; with HKV_OFFLOAD_DYNAMIC those of the dynamic units are laid out in the host buffer
+  // (their offsets stay relative to that buffer until hkv_compress_offload knows both addresses)
+  int64_t hoff = 0;
   for (auto& u : c.units) {
-    u.k_off = off;  off = align_up(off + static_cast<int64_t>(kRowBytes) * u.plane_rows);
-    u.v_off = off;  off = align_up(off + static_cast<int64_t>(kRowBytes) * u.plane_rows);
+    int64_t& o = (offload && u.type == 1) ? hoff : off;
+    u.k_off = o;  o = align_up(o + static_cast<int64_t>(kRowBytes) * u.plane_rows);
+    u.v_off = o;  o = align_up(o + static_cast<int64_t>(kRowBytes) * u.plane_rows);
   }
   c.cache_bytes = static_cast<size_t>(off);
+  c.host_bytes = static_cast<size_t>(hoff);
 
   // ---- workspace layout: s_w per static unit, then the row statistics of the window softmax ----
   int64_t woff = 0;
@@ -150,25 +158,38 @@ hkv_status d2h(void* dst, const void* src, size_t bytes, cudaStream_t s) {
 
 extern "C" {
 
-hkv_status hkv_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type, const int32_t* budgets,
-                    size_t* cache_bytes, size_t* workspace_bytes) {
+static hkv_status plan_common(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type,
+                              const int32_t* budgets, size_t* cache_bytes, size_t* workspace_bytes, size_t* host_bytes) {
   if (!cache_bytes || !workspace_bytes) return HKV_ERR_INVALID_ARG;
   try {
     hkv_cache tmp;
-    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, tmp, nullptr, nullptr);
+    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, tmp, nullptr, nullptr, host_bytes != nullptr);
     if (st != HKV_OK) return st;
     *cache_bytes = tmp.cache_bytes;
     *workspace_bytes = tmp.workspace_bytes;
+    if (host_bytes) *host_bytes = tmp.host_bytes;
     return HKV_OK;
   } catch (...) {
     return HKV_ERR_INVALID_ARG;
   }
 }
 
-hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
-                        const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
-                        const uint8_t* head_type, const int32_t* budgets, void* cache_mem, size_t cache_bytes,
-                        void* workspace, size_t workspace_bytes, void* stream, hkv_cache** out) {
+hkv_status hkv_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type, const int32_t* budgets,
+                    size_t* cache_bytes, size_t* workspace_bytes) {
+  return plan_common(cfg, seq_lens, head_type, budgets, cache_bytes, workspace_bytes, nullptr);
+}
+
+hkv_status hkv_plan_offload(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type,
+                            const int32_t* budgets, size_t* cache_bytes, size_t* workspace_bytes, size_t* host_bytes) {
+  if (!host_bytes) return HKV_ERR_INVALID_ARG;
+  return plan_common(cfg, seq_lens, head_type, budgets, cache_bytes, workspace_bytes, host_bytes);
+}
+
+static hkv_status compress_common(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                                  const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                                  const uint8_t* head_type, const int32_t* budgets, void* cache_mem, size_t cache_bytes,
+                                  void* host_mem, size_t host_bytes, bool offload, void* workspace,
+                                  size_t workspace_bytes, void* stream, hkv_cache** out) {
   if (!out) return HKV_ERR_INVALID_ARG;
   *out = nullptr;
   if (!k || !v || !is_text || !cache_mem || !workspace) return HKV_ERR_INVALID_ARG;
@@ -177,7 +198,31 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
     c = new hkv_cache();
     int64_t ws_rowstat_off = 0;
     int tiles_max = 0;
-    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, *c, &ws_rowstat_off, &tiles_max);
+    hkv_status st = build_plan(cfg, seq_lens, head_type, budgets, *c, &ws_rowstat_off, &tiles_max, offload);
+    if (st == HKV_OK && offload) {
+      if (c->host_bytes > 0 && !host_mem) st = HKV_ERR_INVALID_ARG;
+      else if (host_bytes < c->host_bytes || (reinterpret_cast<uintptr_t>(host_mem) & (kAlign - 1))) st = HKV_ERR_WORKSPACE;
+      if (st == HKV_OK && c->host_bytes > 0) {
+        // the device must reach the whole buffer at the very pointer values given: pinned host memory under
+        // unified addressing.  Anything else is refused here rather than found out by a kernel.
+        for (const char* p : {static_cast<const char*>(host_mem), static_cast<const char*>(host_mem) + c->host_bytes - 1}) {
+          cudaPointerAttributes attr;
+          if (cudaPointerGetAttributes(&attr, p) != cudaSuccess || attr.type != cudaMemoryTypeHost ||
+              attr.devicePointer != static_cast<const void*>(p)) {
+            cudaGetLastError();
+            st = HKV_ERR_INVALID_ARG;
+          }
+        }
+      }
+      if (st == HKV_OK) {
+        // the kernels address every plane as cache_mem + offset: the dynamic planes' offsets now span the
+        // distance to the host buffer, which the device reaches at the same (unified) address
+        const int64_t delta = static_cast<int64_t>(reinterpret_cast<intptr_t>(host_mem) -
+                                                   reinterpret_cast<intptr_t>(cache_mem));
+        for (auto& u : c->units)
+          if (u.type == 1) { u.k_off += delta; u.v_off += delta; }
+      }
+    }
     if (st == HKV_OK && c->hdr.n_static > 0 && !q_obs && !token_scores) st = HKV_ERR_INVALID_ARG;
     if (st == HKV_OK && (cache_bytes < c->cache_bytes || workspace_bytes < c->workspace_bytes)) st = HKV_ERR_WORKSPACE;
     if (st == HKV_OK && ((reinterpret_cast<uintptr_t>(cache_mem) | reinterpret_cast<uintptr_t>(workspace)) & (kAlign - 1)))
@@ -221,6 +266,23 @@ hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, con
   }
 }
 
+hkv_status hkv_compress(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                        const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                        const uint8_t* head_type, const int32_t* budgets, void* cache_mem, size_t cache_bytes,
+                        void* workspace, size_t workspace_bytes, void* stream, hkv_cache** out) {
+  return compress_common(cfg, k, v, q_obs, token_scores, is_text, seq_lens, head_type, budgets, cache_mem, cache_bytes,
+                         nullptr, 0, false, workspace, workspace_bytes, stream, out);
+}
+
+hkv_status hkv_compress_offload(const hkv_config* cfg, const void* k, const void* v, const void* q_obs,
+                                const float* token_scores, const uint8_t* is_text, const int32_t* seq_lens,
+                                const uint8_t* head_type, const int32_t* budgets, void* cache_mem, size_t cache_bytes,
+                                void* host_mem, size_t host_bytes, void* workspace, size_t workspace_bytes,
+                                void* stream, hkv_cache** out) {
+  return compress_common(cfg, k, v, q_obs, token_scores, is_text, seq_lens, head_type, budgets, cache_mem, cache_bytes,
+                         host_mem, host_bytes, true, workspace, workspace_bytes, stream, out);
+}
+
 #ifdef HKV_PROFILE
 static unsigned long long* g_prof = nullptr;
 static long long g_prof_ctas = 0, g_prof_cursor = 0;
@@ -249,7 +311,7 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
     const Header& H = c->hdr;
     const Header& H0 = caches[0]->hdr;
     if (H.group != H0.group || H.n_q_heads != H0.n_q_heads || H.n_kv_heads != H0.n_kv_heads ||
-        H.chunk_size != H0.chunk_size || H.scale != H0.scale || ((H.flags ^ H0.flags) & (HKV_OUT_F32 | HKV_GROUP_MAX)))
+        H.chunk_size != H0.chunk_size || H.scale != H0.scale || ((H.flags ^ H0.flags) & (HKV_OUT_F32 | HKV_GROUP_MAX | HKV_OFFLOAD_DYNAMIC)))
       return HKV_ERR_SHAPE;
     P.cache[i] = c->dev_base;
     P.q[i] = q[i];
@@ -267,6 +329,7 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   P.phase = (do_select ? kPhaseSelect : 0u) | (do_attend ? kPhaseAttend : 0u);
   P.out_f32 = (H0.flags & HKV_OUT_F32) ? 1u : 0u;
   P.group_max = (H0.flags & HKV_GROUP_MAX) ? 1u : 0u;
+  P.offload = (H0.flags & HKV_OFFLOAD_DYNAMIC) ? 1u : 0u;
   const int* max_active = nullptr;
   if (decode_cluster_caps(P.group, &max_active) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
   const int total_units = P.unit_prefix[n];

@@ -477,7 +477,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     // the attention's first copies are what the step waits for: start them before anything else
     if (do_attend && !dead) {
       for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
-      if (at_n <= kPrefetchMaxTiles) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
+      if (at_n <= kPrefetchMaxTiles && !P.offload) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
       attn_armed = true;
     }
     // what later calls may ask for (scores, selected ids, attended tokens), off the critical path

@@ -74,6 +74,7 @@ struct DecodeParams {
   uint32_t out_f32;
   uint32_t pdl;        // launched with programmatic stream serialization
   uint32_t group_max;  // chunk score = max over the group's heads instead of their sum
+  uint32_t offload;    // the dynamic units' K/V planes live in host memory: no L2 prefetch requests for them
   int32_t unit_prefix[kMaxMulti + 1];
   char* cache[kMaxMulti];
   const void* q[kMaxMulti];
@@ -119,7 +120,7 @@ struct hkv_cache {
   hkv::Header hdr;
   std::vector<hkv::Unit> units;
   char* dev_base;
-  size_t cache_bytes, workspace_bytes;
+  size_t cache_bytes, workspace_bytes, host_bytes;
   int64_t kv_bytes, summary_bytes, algo_bytes, retained;
   int max_static_rows, max_dyn_rows, max_chunks, max_tiles;
   bool fresh;   // no decode launch has followed the last compression / append yet

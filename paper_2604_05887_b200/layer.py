@@ -29,7 +29,16 @@ class LayerCache:
         self.flags = flags
         self.shape = (L.batch, L.n_q_heads, L.head_dim)
         self.device = device
-        cache_bytes, ws_bytes = hkv.hkv_plan(self.cfg, L.seq_lens, L.head_type, L.budgets)
+        self.host_mem = None
+        if flags & hkv.HKV_OFFLOAD_DYNAMIC:
+            cache_bytes, ws_bytes, host_bytes = hkv.hkv_plan_offload(self.cfg, L.seq_lens, L.head_type, L.budgets)
+            if host_bytes:
+                # 256-byte aligned slice of a pinned buffer the device addresses at the same pointer value
+                raw = torch.empty(host_bytes + 256, dtype=torch.uint8, pin_memory=True)
+                skip = (-raw.data_ptr()) % 256
+                self.host_mem = raw[skip:skip + host_bytes]
+        else:
+            cache_bytes, ws_bytes = hkv.hkv_plan(self.cfg, L.seq_lens, L.head_type, L.budgets)
         self.cache_mem = torch.empty(cache_bytes, dtype=torch.uint8, device=device)
         workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
         k = k_dev if k_dev is not None else to_device_bf16(L.k, device)
@@ -39,8 +48,12 @@ class LayerCache:
         ts = None
         if token_scores is not None:
             ts = torch.from_numpy(np.ascontiguousarray(token_scores, dtype=np.float32)).to(device)
-        self.handle = hkv.hkv_compress(self.cfg, k, v, q_obs, ts, is_text, L.seq_lens, L.head_type, L.budgets,
-                                       self.cache_mem, workspace)
+        if flags & hkv.HKV_OFFLOAD_DYNAMIC:
+            self.handle = hkv.hkv_compress_offload(self.cfg, k, v, q_obs, ts, is_text, L.seq_lens, L.head_type,
+                                                   L.budgets, self.cache_mem, self.host_mem, workspace)
+        else:
+            self.handle = hkv.hkv_compress(self.cfg, k, v, q_obs, ts, is_text, L.seq_lens, L.head_type, L.budgets,
+                                           self.cache_mem, workspace)
         self.workspace = workspace if keep_workspace else None
         if not keep_workspace:
             torch.cuda.current_stream().synchronize()   # inputs and workspace are released below

@@ -36,8 +36,10 @@ def test_oracle_append_equals_compressing_the_longer_sequence_for_dynamic_heads(
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("cs,C,budget,cap", [(16, 500, 0.2, 40), (32, 1000, 1.0, 70), (8, 333, 0.5, 19), (64, 700, 0.1, 130)])
-def test_append_matches_oracle_step_by_step(cs, C, budget, cap):
+@pytest.mark.parametrize("cs,C,budget,cap,offload", [(16, 500, 0.2, 40, False), (32, 1000, 1.0, 70, False),
+                                                     (8, 333, 0.5, 19, False), (64, 700, 0.1, 130, False),
+                                                     (16, 450, 0.3, 25, True)])
+def test_append_matches_oracle_step_by_step(cs, C, budget, cap, offload):
     import parity_util as P
     from paper_2604_05887_b200 import binding as hkv
     from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
@@ -45,7 +47,7 @@ def test_append_matches_oracle_step_by_step(cs, C, budget, cap):
     if budget >= 1.0:
         L.budgets[:] = 10 ** 6                                   # "everything", also after the sequence has grown
     L = _with_room(L, cap)
-    lc = LayerCache(L, flags=hkv.HKV_OUT_F32, append_capacity=cap)
+    lc = LayerCache(L, flags=hkv.HKV_OUT_F32 | (hkv.HKV_OFFLOAD_DYNAMIC if offload else 0), append_capacity=cap)
     oc = o.compress_layer(L)
     rng = np.random.default_rng(cs)
     G = L.group

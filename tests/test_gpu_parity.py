@@ -117,6 +117,37 @@ def test_group_max_scoring_variant(P, Hq, Hkv):
     assert rep["stats"]["n_dynamic"] == 2 * Hkv
 
 
+def test_offloaded_dynamic_heads_variant(P):
+    """HKV_OFFLOAD_DYNAMIC: the dynamic heads' K/V planes sit in pinned host memory; same results, two steps."""
+    from paper_2604_05887_b200 import binding as hkv
+    L = small(B=2, C=1300, cs=16, w=8, budget=0.2, n_steps=2)
+    rep = P.compare_layer(L, flags=hkv.HKV_OUT_F32 | hkv.HKV_OFFLOAD_DYNAMIC)
+    assert rep["stats"]["n_dynamic"] > 0
+    # all static: no host buffer at all
+    Ls = small(B=1, C=600, cs=16, w=8, budget=0.2, n_steps=1, head_type=np.zeros((1, 4), np.uint8))
+    P.compare_layer(Ls, flags=hkv.HKV_OUT_F32 | hkv.HKV_OFFLOAD_DYNAMIC)
+    # the plain entry points refuse the flag, the offload ones its absence, and device memory is not host memory
+    cfg = hkv.make_config(L.batch, L.n_q_heads, L.n_kv_heads, 128, L.max_seq_len, 16, 8, 0.0, hkv.HKV_OFFLOAD_DYNAMIC, 0)
+    with pytest.raises(hkv.HkvError):
+        hkv.hkv_plan(cfg, L.seq_lens, L.head_type, L.budgets)
+    cfg0 = hkv.make_config(L.batch, L.n_q_heads, L.n_kv_heads, 128, L.max_seq_len, 16, 8, 0.0, 0, 0)
+    with pytest.raises(hkv.HkvError):
+        hkv.hkv_plan_offload(cfg0, L.seq_lens, L.head_type, L.budgets)
+    cb, wb, hb = hkv.hkv_plan_offload(cfg, L.seq_lens, L.head_type, L.budgets)
+    assert hb > 0 and hb % 256 == 0
+    import torch
+    dev_buf = torch.empty(hb, dtype=torch.uint8, device="cuda")
+    z = torch.zeros(8, dtype=torch.uint8, device="cuda")
+    st = hkv.lib.hkv_compress_offload(hkv.C.byref(cfg), z.data_ptr(), z.data_ptr(), z.data_ptr(), None, z.data_ptr(),
+                                      hkv._ptr(hkv._i32(L.seq_lens), hkv.C.c_int32),
+                                      hkv._ptr(hkv._u8(L.head_type), hkv.C.c_uint8),
+                                      hkv._ptr(hkv._i32(L.budgets), hkv.C.c_int32),
+                                      torch.empty(cb, dtype=torch.uint8, device="cuda").data_ptr(), cb,
+                                      dev_buf.data_ptr(), hb, torch.empty(wb, dtype=torch.uint8, device="cuda").data_ptr(),
+                                      wb, None, hkv.C.byref(hkv.C.c_void_p(None)))
+    assert st == 1        # HKV_ERR_INVALID_ARG before anything is launched
+
+
 def test_second_geometry_qwen25_vl_3b(P):
     """16 query / 2 KV heads (group of 8), head_dim 128: the smaller model the paper also evaluates."""
     L = small(B=3, C=5000, cs=32, w=32, Hq=16, Hkv=2, budget=0.1, n_steps=2)
