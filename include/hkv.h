@@ -17,9 +17,11 @@
  *
  * Conventions
  *   - plain C linkage; no exception crosses the boundary; every call returns a status.  Argument
- *     errors are found on the host before anything is launched.  Global state is limited to what
- *     two entry points document: the helper stream of hkv_decode_step_host and the fixed scratch of
- *     hkv_topk_chunks_noalloc.
+ *     errors are found on the host before anything is launched.  Global state is limited to a
+ *     helper stream with a few events per device (hkv_compress builds the dynamic heads on it beside
+ *     the static ones, hkv_decode_step_host runs its copies on it; both fork it from and join it to
+ *     the caller's stream, so the caller sees one ordered stream and may capture the calls in a
+ *     graph) and the fixed scratch of hkv_topk_chunks_noalloc.
  *   - "dev" pointers are device (HBM) addresses on the current CUDA device, "host" pointers are
  *     ordinary host memory.  bf16 tensors are passed as void*.
  *   - the caller owns every device buffer, including cache_mem and workspace.  The library never

@@ -158,6 +158,42 @@ hkv_status d2h(void* dst, const void* src, size_t bytes, cudaStream_t s) {
 
 extern "C" {
 
+namespace {
+// A second stream and a few events per device, created on first use and never destroyed.
+// hkv_decode_step_host: the queries of the layers after the first travel to the device while the
+// first layer runs, and the outputs of all but the last group of layers travel back while later
+// layers run.  hkv_compress: the dynamic heads' planes and chunk means are built beside the static
+// heads' window scores, selection and gather (independent work on disjoint memory).
+constexpr int kStepGroups = 4;
+struct StepSide {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, q_done = nullptr, q_done2 = nullptr, join = nullptr, out[kStepGroups] = {};
+  bool ready = false;
+  std::mutex enqueue;   // held while a call records and waits on these events, so that host threads do not interleave
+};
+StepSide g_step_side[64];
+std::mutex g_step_mutex;
+
+StepSide* step_side() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_step_mutex);
+  StepSide& s = g_step_side[dev];
+  if (!s.ready) {
+    bool ok = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.q_done, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.q_done2, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kStepGroups; ++i)
+      ok = cudaEventCreateWithFlags(&s.out[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return nullptr; }
+    s.ready = true;
+  }
+  return &s;
+}
+}  // namespace
+
 static hkv_status plan_common(const hkv_config* cfg, const int32_t* seq_lens, const uint8_t* head_type,
                               const int32_t* budgets, size_t* cache_bytes, size_t* workspace_bytes, size_t* host_bytes) {
   if (!cache_bytes || !workspace_bytes) return HKV_ERR_INVALID_ARG;
@@ -248,6 +284,15 @@ static hkv_status compress_common(const hkv_config* cfg, const void* k, const vo
     // n_valid and the error word start at zero
     ok = ok && cudaMemsetAsync(c->dev_base + H.n_valid_off, 0, static_cast<size_t>(H.err_off + 8 - H.n_valid_off), s) ==
                    cudaSuccess;
+    // dynamic heads beside the static ones, on the library's second stream (forked from and joined to `s`)
+    StepSide* side = (H.n_static > 0 && H.n_dynamic > 0) ? step_side() : nullptr;
+    std::unique_lock<std::mutex> side_lock;
+    if (side) side_lock = std::unique_lock<std::mutex>(side->enqueue);
+    if (ok && side) {
+      ok = cudaEventRecord(side->fork, s) == cudaSuccess && cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess;
+      ok = ok && launch_build_dynamic(c->dev_base, k, v, H, c->max_dyn_rows, c->max_chunks, side->stream) == cudaSuccess;
+      ok = ok && cudaEventRecord(side->join, side->stream) == cudaSuccess;
+    }
     if (ok && H.n_static > 0) {
       if (!token_scores)
         ok = launch_window_scores(c->dev_base, static_cast<char*>(workspace), k, q_obs, H, c->units, ws_rowstat_off,
@@ -255,8 +300,9 @@ static hkv_status compress_common(const hkv_config* cfg, const void* k, const vo
       ok = ok && launch_static_select(c->dev_base, static_cast<char*>(workspace), token_scores, is_text, H, s) == cudaSuccess;
       ok = ok && launch_gather_static(c->dev_base, k, v, H, c->max_static_rows, s) == cudaSuccess;
     }
-    if (ok && H.n_dynamic > 0)
+    if (ok && H.n_dynamic > 0 && !side)
       ok = launch_build_dynamic(c->dev_base, k, v, H, c->max_dyn_rows, c->max_chunks, s) == cudaSuccess;
+    if (ok && side) ok = cudaStreamWaitEvent(s, side->join, 0) == cudaSuccess;
     if (!ok) { cudaGetLastError(); delete c; return HKV_ERR_CUDA; }
     *out = c;
     return HKV_OK;
@@ -399,39 +445,6 @@ hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_
   return HKV_OK;
 }
 
-namespace {
-// A second stream and a few events per device for hkv_decode_step_host: the queries of the layers
-// after the first travel to the device while the first layer runs, and the outputs of all but the
-// last group of layers travel back while later layers run.  Created on first use, never destroyed.
-constexpr int kStepGroups = 4;
-struct StepSide {
-  cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, q_done = nullptr, q_done2 = nullptr, join = nullptr, out[kStepGroups] = {};
-  bool ready = false;
-};
-StepSide g_step_side[64];
-std::mutex g_step_mutex;
-
-StepSide* step_side() {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  std::lock_guard<std::mutex> lock(g_step_mutex);
-  StepSide& s = g_step_side[dev];
-  if (!s.ready) {
-    bool ok = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&s.q_done, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&s.q_done2, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; ok && i < kStepGroups; ++i)
-      ok = cudaEventCreateWithFlags(&s.out[i], cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return nullptr; }
-    s.ready = true;
-  }
-  return &s;
-}
-}  // namespace
-
 hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void* q_host, void* out_host, void* q_dev,
                                 void* out_dev, void* stream) {
   if (!caches || n < 1 || !q_host || !out_host || !q_dev || !out_dev) return HKV_ERR_INVALID_ARG;
@@ -450,6 +463,8 @@ hkv_status hkv_decode_step_host(hkv_cache* const* caches, int32_t n, const void*
   char* oh = static_cast<char*>(out_host);
   char* od = static_cast<char*>(out_dev);
   StepSide* side = n >= 2 ? step_side() : nullptr;
+  std::unique_lock<std::mutex> side_lock;
+  if (side) side_lock = std::unique_lock<std::mutex>(side->enqueue);
   const int q_split = std::min(n, 4);   // layers 1 .. q_split - 1 get their queries in a first, short transfer
   bool ok = true;
   auto cu = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
