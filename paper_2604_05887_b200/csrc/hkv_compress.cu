@@ -244,12 +244,28 @@ __global__ void __launch_bounds__(kKeepThreads)
 
   if (tid == 0) s_ntext = 0;
   __syncthreads();
+  // four tokens per thread and step when the rows of is_text and of the scores start on 4-token boundaries
+  const bool vec = cached && (hdr->max_seq_len & 3) == 0 && (reinterpret_cast<uintptr_t>(is_text) & 3) == 0 &&
+                   (reinterpret_cast<uintptr_t>(scores) & 15) == 0;
   int cnt = 0;
+  if (vec) {
+#pragma unroll 8
+    for (int i = 4 * tid; i < hist_end; i += 4 * kKeepThreads) {
+      const uchar4 t4 = *reinterpret_cast<const uchar4*>(txt + i);
+      uint4 f = make_uint4(t4.x != 0, t4.y != 0, t4.z != 0, t4.w != 0);
+      if (i + 1 >= hist_end) f.y = 0u;   // the tokens of the window are not counted
+      if (i + 2 >= hist_end) f.z = 0u;
+      if (i + 3 >= hist_end) f.w = 0u;
+      cnt += static_cast<int>(f.x + f.y + f.z + f.w);
+      *reinterpret_cast<uint4*>(skey + i) = f;
+    }
+  } else {
 #pragma unroll 16
-  for (int i = tid; i < hist_end; i += kKeepThreads) {
-    const int t = txt[i] != 0;
-    cnt += t;
-    if (cached) skey[i] = static_cast<uint32_t>(t);
+    for (int i = tid; i < hist_end; i += kKeepThreads) {
+      const int t = txt[i] != 0;
+      cnt += t;
+      if (cached) skey[i] = static_cast<uint32_t>(t);
+    }
   }
   for (int off = 16; off >= 1; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
   if ((tid & 31) == 0 && cnt) atomicAdd(&s_ntext, cnt);
@@ -268,14 +284,23 @@ __global__ void __launch_bounds__(kKeepThreads)
     if (cached) {
       // each token's role once: kKeepAlways = kept regardless, 0 = out of the ranking, else its score's key
       // (a thread rewrites only the entries it flagged above)
-#pragma unroll 16
-      for (int i = tid; i < C; i += kKeepThreads) {
-        uint32_t key = kKeepAlways;
-        if (i < hist_end) {
-          const bool is_t = skey[i] != 0u;
-          key = (is_t == rank_text) ? float_key(scores[i]) : (is_t ? kKeepAlways : 0u);
+      auto role = [&](int i, uint32_t flag, float score) {
+        if (i >= hist_end) return kKeepAlways;
+        const bool is_t = flag != 0u;
+        return (is_t == rank_text) ? float_key(score) : (is_t ? kKeepAlways : 0u);
+      };
+      if (vec) {
+        // (the rows are max_seq_len floats long, so a whole float4 is readable wherever its first token is)
+#pragma unroll 8
+        for (int i = 4 * tid; i < C; i += 4 * kKeepThreads) {
+          const float4 sc4 = *reinterpret_cast<const float4*>(scores + i);
+          const uint4 f = i < hist_end ? *reinterpret_cast<const uint4*>(skey + i) : make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(skey + i) =
+              make_uint4(role(i, f.x, sc4.x), role(i + 1, f.y, sc4.y), role(i + 2, f.z, sc4.z), role(i + 3, f.w, sc4.w));
         }
-        skey[i] = key;
+      } else {
+#pragma unroll 16
+        for (int i = tid; i < C; i += kKeepThreads) skey[i] = role(i, i < hist_end ? skey[i] : 0u, i < hist_end ? scores[i] : 0.f);
       }
       __syncthreads();
       emitted = block_topk_keyed<kKeepThreads>(
