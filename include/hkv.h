@@ -319,10 +319,11 @@ hkv_status hkv_window_scores_offset(const hkv_cache* cache, int32_t b, int32_t h
 
 hkv_status hkv_cache_stats(const hkv_cache* cache, hkv_stats* stats);
 
-/* How many thread-block clusters of 1, 2, 4, 8 and 16 CTAs of the decode kernel (for a group of
- * `group` query heads per KV head) the current device can hold at once: max_active_clusters[0..4].
- * hkv_decode_attn picks, per launch, the largest cluster size whose capacity covers all (sequence,
- * KV head) units of the launch (Appendix A's per-head work is what a cluster owns).  Needs a device. */
+/* How many thread-block clusters of 1, 2, ..., 16 CTAs of the decode kernel (for a group of `group`
+ * query heads per KV head) the current device can hold at once: max_active_clusters[c - 1] for size
+ * c, 16 entries.  hkv_decode_attn picks, per launch, the largest even cluster size (or 1) whose
+ * capacity covers all (sequence, KV head) units of the launch and that leaves every CTA at least
+ * two tiles (Appendix A's per-head work is what a cluster owns).  Needs a device. */
 hkv_status hkv_decode_cluster_capacity(int32_t group, int32_t* max_active_clusters);
 
 /* Device error word: code is HKV_OK, HKV_ERR_TIMEOUT or HKV_ERR_INDEX; detail identifies the place.

@@ -298,9 +298,9 @@ def hkv_window_scores_offset(cache: int, b: int, h: int) -> int:
 
 def hkv_decode_cluster_capacity(group: int) -> dict:
     """{cluster size: clusters of the decode kernel the current device holds at once}."""
-    out = np.zeros(5, dtype=np.int32)
+    out = np.zeros(16, dtype=np.int32)
     _check(lib.hkv_decode_cluster_capacity(int(group), _ptr(out, C.c_int32)), "hkv_decode_cluster_capacity")
-    return {1 << i: int(out[i]) for i in range(5)}
+    return {i + 1: int(out[i]) for i in range(16)}
 
 
 HKV_BUDGET_PAD_POW2 = 1

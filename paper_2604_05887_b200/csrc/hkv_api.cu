@@ -610,7 +610,7 @@ hkv_status hkv_decode_cluster_capacity(int32_t group, int32_t* max_active_cluste
   if (!max_active_clusters || group < 1 || group > kMaxGroup) return HKV_ERR_INVALID_ARG;
   const int* caps = nullptr;
   if (decode_cluster_caps(group, &caps) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
-  for (int i = 0, c = 1; c <= kMaxCluster; c <<= 1, ++i) max_active_clusters[i] = caps[c];
+  for (int c = 1; c <= kMaxCluster; ++c) max_active_clusters[c - 1] = caps[c];
   return HKV_OK;
 }
 
@@ -631,7 +631,8 @@ hkv_status hkv_cache_stats(const hkv_cache* c, hkv_stats* st) {
     int assumed[kMaxCluster + 1] = {};
     if (decode_cluster_caps(c->hdr.group, &max_active) != cudaSuccess) {
       cudaGetLastError();
-      for (int k = 1; k <= kMaxCluster; k <<= 1) assumed[k] = 2 * 148 / k;
+      static const int b200[kMaxCluster + 1] = {0, 296, 148, 93, 71, 56, 45, 37, 33, 30, 26, 21, 21, 17, 14, 14, 14};
+      for (int k = 1; k <= kMaxCluster; ++k) assumed[k] = b200[k];   // as measured on a B200 (148 SMs, two CTAs each)
       max_active = assumed;
     }
     st->n_splits = c->hdr.n_units * choose_cluster(c->hdr.n_units, c->max_tiles, max_active);

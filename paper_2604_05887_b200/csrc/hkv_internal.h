@@ -95,7 +95,7 @@ constexpr int kDecCtasPerSm = 2;
 
 // ---- kernel launchers (definitions in the .cu files) ----
 // Picks the cluster size for `total_units` units whose longest token list has `max_tiles` tiles;
-// max_active[c] = clusters of c CTAs the device holds at once (index 1, 2, 4, 8, 16).
+// max_active[c] = clusters of c CTAs the device holds at once (index 1 .. kMaxCluster).
 int choose_cluster(int total_units, int max_tiles, const int* max_active);
 // Cluster capacities of the decode kernel for this group size (also performs the kernel's one-time
 // set-up; call before the first launch_decode).

@@ -346,15 +346,19 @@ def test_more_units_than_clusters_fit(P):
 
 
 def test_unit_counts_that_select_every_cluster_size(P):
-    """1, 2, 4, 8 and 16 CTAs per unit (the launch picks the largest size that fits all units in one wave)."""
+    """1, 2, 4, 6, 8, 10, 12, 14 or 16 CTAs per unit: the launch picks the largest even size (or 1) that fits all
+    units in one wave and leaves a CTA two tiles; sizes need not be powers of two."""
     from paper_2604_05887_b200 import binding as hkv
     caps = hkv.hkv_decode_cluster_capacity(7)
     seen = set()
-    for B in (1, 3, 6, 12, 30, 50):
-        L = small(B=B, C=1500, cs=32, w=8, budget=0.5, n_steps=1, ragged=False)
+    for B in (1, 4, 6, 8, 10, 12, 30, 50):
+        L = small(B=B, C=2200, cs=32, w=8, budget=0.5, n_steps=1, ragged=False)
         rep = P.compare_layer(L, units=[(0, 0), (B - 1, 3), (B // 2, 1), (B // 2, 2)])
-        seen.add(rep["stats"]["n_splits"] // (4 * B))
-    assert seen >= {1, 2, 4, 8}, (seen, caps)
+        size = rep["stats"]["n_splits"] // (4 * B)
+        want = max([1] + [c for c in range(2, 17, 2) if caps[c] >= 4 * B and 2 * c <= (1100 + 31) // 32])
+        assert size == want, (B, size, want, caps)
+        seen.add(size)
+    assert len(seen) >= 6 and {1, 2, 4, 8} <= seen, (seen, caps)
 
 
 @pytest.mark.parametrize("case", range(24))
