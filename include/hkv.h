@@ -323,7 +323,8 @@ hkv_status hkv_cache_stats(const hkv_cache* cache, hkv_stats* stats);
  * query heads per KV head) the current device can hold at once: max_active_clusters[c - 1] for size
  * c, 16 entries.  hkv_decode_attn picks, per launch, the largest even cluster size (or 1) whose
  * capacity covers all (sequence, KV head) units of the launch and that leaves every CTA at least
- * two tiles (Appendix A's per-head work is what a cluster owns).  Needs a device. */
+ * two tiles, but no more than ten CTAs per unit when the token lists are short (Appendix A's
+ * per-head work is what a cluster owns).  Needs a device. */
 hkv_status hkv_decode_cluster_capacity(int32_t group, int32_t* max_active_clusters);
 
 /* Device error word: code is HKV_OK, HKV_ERR_TIMEOUT or HKV_ERR_INDEX; detail identifies the place.

@@ -913,14 +913,20 @@ cudaError_t launch_nt(const DecodeParams& params, int total_units, cudaStream_t 
 
 size_t decode_smem_bytes() { return kSmemBytes; }
 
+constexpr int kLatencyCluster = 10;
+
 int choose_cluster(int total_units, int max_tiles, const int* max_active) {
   // The largest even size (or 1) that (a) the device can hold in ONE wave of clusters, (b) leaves every
   // CTA at least two tiles of the longest unit.  max_active[c] = clusters of size c resident at once.
   // Even sizes only: two CTAs share an SM, and an odd cluster leaves half an SM idle (measured: 13 CTAs
   // per unit are slower than 12).  Sizes need not be powers of two.
+  // Short lists (at most 16 tiles per CTA at ten CTAs per unit) are bound by the step's chain of latencies,
+  // not by bandwidth; there ten CTAs per unit measured best at every batch size tried (1 .. 6 sequences of
+  // four KV heads), larger clusters paying more for their barriers and exchanges than they gain.
   int c = 1;
   for (int t = 2; t <= kMaxCluster; t += 2)
     if (max_active[t] >= total_units && t * 2 <= max_tiles) c = t;
+  if (c > kLatencyCluster && max_tiles <= kLatencyCluster * 16) c = kLatencyCluster;
   return c;
 }
 

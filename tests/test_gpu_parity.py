@@ -345,20 +345,30 @@ def test_more_units_than_clusters_fit(P):
     assert rep["stats"]["n_splits"] == 200
 
 
+def _expected_cluster(caps, units, tiles):
+    c = max([1] + [t for t in range(2, 17, 2) if caps[t] >= units and 2 * t <= tiles])
+    return 10 if c > 10 and tiles <= 160 else c
+
+
 def test_unit_counts_that_select_every_cluster_size(P):
-    """1, 2, 4, 6, 8, 10, 12, 14 or 16 CTAs per unit: the launch picks the largest even size (or 1) that fits all
-    units in one wave and leaves a CTA two tiles; sizes need not be powers of two."""
+    """1, 2, 4, 6, 8, 10, 12 or 16 CTAs per unit: the launch picks the largest even size (or 1) that fits all units
+    in one wave and leaves a CTA two tiles, capped at 10 for short token lists; sizes need not be powers of two."""
     from paper_2604_05887_b200 import binding as hkv
     caps = hkv.hkv_decode_cluster_capacity(7)
     seen = set()
-    for B in (1, 4, 6, 8, 10, 12, 30, 50):
+    for B in (1, 6, 8, 10, 12, 30, 50):
         L = small(B=B, C=2200, cs=32, w=8, budget=0.5, n_steps=1, ragged=False)
         rep = P.compare_layer(L, units=[(0, 0), (B - 1, 3), (B // 2, 1), (B // 2, 2)])
         size = rep["stats"]["n_splits"] // (4 * B)
-        want = max([1] + [c for c in range(2, 17, 2) if caps[c] >= 4 * B and 2 * c <= (1100 + 31) // 32])
-        assert size == want, (B, size, want, caps)
+        assert size == _expected_cluster(caps, 4 * B, (1100 + 31) // 32), (B, size, caps)
         seen.add(size)
-    assert len(seen) >= 6 and {1, 2, 4, 8} <= seen, (seen, caps)
+    for B in (1, 4):                       # long lists (188 tiles per unit): the cap does not apply
+        L = small(B=B, C=6000, cs=32, w=8, budget=1.0, n_steps=1, ragged=False)
+        rep = P.compare_layer(L, units=[(0, 0), (B - 1, 3)])
+        size = rep["stats"]["n_splits"] // (4 * B)
+        assert size == _expected_cluster(caps, 4 * B, (6000 + 31) // 32), (B, size, caps)
+        seen.add(size)
+    assert {1, 2, 4, 6, 8, 10, 12, 16} <= seen, (seen, caps)
 
 
 @pytest.mark.parametrize("case", range(24))
