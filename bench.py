@@ -392,6 +392,8 @@ def main():
                     help="skip the extra per-launch measurement of the single-layer 32K sweep cell (cfg4)")
     ap.add_argument("--sweep", action="store_true", help="run the 100-cell single-layer sweep (cfg4) instead of the step benchmark")
     ap.add_argument("--sweep-quick", action="store_true", help="with --sweep: only budgets 10 % and 100 % at static fraction 0.5")
+    ap.add_argument("--next-rows", action="store_true",
+                    help="time hkv_classify_heads and the host-offload variant on layer 0 even in a reduced (--layers) run")
     ap.add_argument("--layers", type=int, default=0,
                     help="use only the first N layers of the workload (small case for profiler captures; "
                          "the line is then marked reduced and is not the headline number)")
@@ -597,6 +599,8 @@ def main():
         del caches, qs, outs
         torch.cuda.empty_cache()
         line["other_workloads"] = [measure_other_workload("cfg4", 4, args.seed + 4, dev, peak)]
+        line["next_rows"] = [measure_classification(L0, dev), measure_offload(L0, dev)]
+    elif rank == 0 and world == 1 and args.next_rows:
         line["next_rows"] = [measure_classification(L0, dev), measure_offload(L0, dev)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt, n = oracle_decode_timing(L0, args.cpu_seconds)
