@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       float acc = 0.f, acc2 = 0.f, acc3 = 0.f, acc4 = 0.f;
       if (row0 + 128 * half < R) {                     // same for the whole warp
         groups([&](int g, float (&v)[32]) {
+          if (row0 + 128 * half + 32 * g >= R) return;   // 32 padding rows: nothing to add (same for the whole warp)
           const float4* info = rowinfo + 128 * half + 32 * g;
           if (all_visible) {
 #pragma unroll
