@@ -131,6 +131,14 @@ def test_gpu_classify_topk_counts(fraction):
 
 
 @pytest.mark.gpu
+def test_gpu_classify_several_row_blocks_in_one_pass():
+    """420 rows per unit in one pass: two resident 256-row blocks per key range (the second partly padding)."""
+    L = hi.tiny(seed=36, B=2, C=1400, chunk_size=32, w=8, Hq=28, Hkv=4, d=128)
+    _check_case(L, 60, 0.05)
+    _check_case(L, 60, 0.05, workspace="min")
+
+
+@pytest.mark.gpu
 def test_gpu_classify_rows_longer_than_shared_memory():
     L = hi.tiny(seed=33, B=1, C=50021, chunk_size=32, w=8, Hq=8, Hkv=2, d=128)
     _check_case(L, 3, 0.05)
