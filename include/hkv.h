@@ -20,8 +20,9 @@
  *     errors are found on the host before anything is launched.  Global state is limited to a
  *     helper stream with a few events per device (hkv_compress builds the dynamic heads on it beside
  *     the static ones, hkv_decode_step_host runs its copies on it; both fork it from and join it to
- *     the caller's stream, so the caller sees one ordered stream and may capture the calls in a
- *     graph) and the fixed scratch of hkv_topk_chunks_noalloc.
+ *     the caller's stream, so the caller sees one ordered stream) and the fixed scratch of
+ *     hkv_topk_chunks_noalloc.  hkv_compress uploads its plan from ordinary host memory that it frees
+ *     on return, so it is not a call to capture in a CUDA graph; the decode calls are.
  *   - "dev" pointers are device (HBM) addresses on the current CUDA device, "host" pointers are
  *     ordinary host memory.  bf16 tensors are passed as void*.
  *   - the caller owns every device buffer, including cache_mem and workspace.  The library never
