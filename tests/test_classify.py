@@ -173,3 +173,19 @@ def test_gpu_classify_uniform_rows_and_errors():
         with pytest.raises(hkv.HkvError) as e:
             hkv.hkv_classify_heads(cfg, k, q, a["seq_lens"], a["n_text"], a["fraction"], 0.9, a["ws"], sc, ty)
         assert e.value.status == status
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", range(10))
+def test_gpu_classify_random_shapes(case):
+    """Seeded random geometry: batch, lengths, group size, text-token counts, top-k fraction, workspace size."""
+    rng = np.random.default_rng(7000 + case)
+    Hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 7, 8, 16]))
+    B = int(rng.integers(1, 5))
+    C = int(rng.integers(40, 6000))
+    T = int(rng.integers(1, 80))
+    fraction = float(rng.choice([0.01, 0.05, 0.05, 0.2, 0.5]))
+    L = hi.tiny(seed=7100 + case, B=B, C=C, chunk_size=32, w=8, Hq=G * Hkv, Hkv=Hkv, d=128,
+                ragged=bool(rng.integers(0, 2)) and C > 5 * B + 16)
+    _check_case(L, T, fraction, workspace=str(rng.choice(["preferred", "min"])), seed=case)
