@@ -136,7 +136,7 @@ hkv_status build_plan(const hkv_config* cfg, const int32_t* seq_lens, const uint
     if (u.type == 0) { u.ws_scores_off = woff; woff = align_up(woff + 4ll * u.C); }
   }
   const int R = w * G, Rpad = (R + 15) / 16 * 16;
-  const int tiles_max = (max_C + 63) / 64;
+  const int tiles_max = 2 * ((max_C + 127) / 128);   // two partial row statistics per 128-key tile at most
   if (ws_rowstat_off) *ws_rowstat_off = woff;
   if (n_col_tiles_max) *n_col_tiles_max = tiles_max;
   woff = align_up(woff + 8ll * H.n_static * tiles_max * Rpad + 8ll * H.n_static * Rpad);

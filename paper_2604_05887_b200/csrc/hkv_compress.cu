@@ -29,10 +29,10 @@ __device__ __forceinline__ const Unit* unit_of(const char* cache, const Header* 
 // tensor cores: one CTA = one static unit x one range of 128-key tiles x one block of up to 256
 // rows; the row block stays in shared memory, the key tiles stream; logits in base 2.
 // MODE 0: accumulator rows = window rows; a draining thread owns one row and keeps its running
-//         (max, exp-sum) over the CTA's keys; stats: float2 [n_static][n_ranges_max][Rpad].
+//         (max, exp-sum) over its half of the CTA's keys; stats: float2 [n_static][2 ranges][Rpad].
 // MODE 1: with the rows' final (max, sum) known, accumulator rows = keys; a draining thread owns
-//         one key and sums the normalised probabilities of its half of the rows, the two halves
-//         meet in shared memory, and s_w[key] (+)= sum / R (written by the first row block, added
+//         one key and sums the normalised probabilities of its quarter of the rows, the four
+//         quarters meet in shared memory, and s_w[key] (+)= sum / R (written by the first row block, added
 //         to by later ones).
 // grid (key ranges, n_static).
 // ---------------------------------------------------------------------------------------------
@@ -68,15 +68,18 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
   if (MODE == 0) {
     float m_run = -INFINITY, z_run = 0.f;
     int my_row = -1;
-    auto epilogue = [&](int tile, int lane_row, int half, auto groups, float*, float*, uint64_t*) {
-      const int r = row0 + 128 * half + lane_row;
+    int my_half = 0;
+    auto epilogue = [&](int tile, int lane_row, int part, auto groups, float*, auto, uint64_t*) {
+      // accumulator columns 64 part .. + 63 = keys 64 (part & 1) .. + 63 of the tile for the rows of block part >> 1
+      const int r = row0 + 128 * (part >> 1) + lane_row;
       my_row = r;
-      if (row0 + 128 * half + (lane_row & ~31) >= R) return;   // the warp's rows are all padding
+      my_half = part & 1;
+      if (row0 + 128 * (part >> 1) + (lane_row & ~31) >= R) return;   // the warp's rows are all padding
       const int lim = causal ? (C - w + r / G) : (C - 1);      // last key the row sees
       const int j0 = tile * tc::kKeysPerTile;
       const bool all_visible = j0 + tc::kKeysPerTile - 1 <= (causal ? C - w : C - 1);   // to every row
       groups([&](int g, float (&v)[32]) {
-        const int jg = j0 + g * 32;
+        const int jg = j0 + 64 * (part & 1) + g * 32;
         float gmax = -INFINITY;
         if (all_visible) {
           float g0 = v[0], g1 = v[1], g2 = v[2], g3 = v[3];   // four short chains instead of one long one
@@ -111,8 +114,10 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       });
     };
     const bool ok = tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue);
+    // two threads share a row (one per half of every tile): two partial statistics per key range
     if (threadIdx.x >= 64 && my_row >= 0 && my_row < R)
-      stats[(static_cast<size_t>(blockIdx.y) * n_ranges_max + blockIdx.x) * Rpad + my_row] = make_float2(m_run, z_run);
+      stats[(static_cast<size_t>(blockIdx.y) * n_ranges_max + 2 * blockIdx.x + my_half) * Rpad + my_row] =
+          make_float2(m_run, z_run);
     if (!ok && threadIdx.x == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrScoreWait; }
   } else {
     for (int i = threadIdx.x; i < tc::kQRows; i += tc::kThreads) {
@@ -129,16 +134,17 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
     const float inv_R = 1.f / static_cast<float>(R);
     int n_done = 0;
     bool pair_ok = true;
-    auto epilogue = [&](int tile, int lane_row, int half, auto groups, float* scratch, float* partner,
+    auto epilogue = [&](int tile, int lane_row, int part, auto groups, float* scratch, auto siblings,
                         uint64_t* pair_bar) {
+      // accumulator columns 64 part .. + 63 = window rows row0 + 64 part + (0..63) for the key of this lane
       const int j0 = tile * tc::kKeysPerTile, j = j0 + lane_row;
       const float jf = static_cast<float>(j);
       const bool all_visible = j0 + tc::kKeysPerTile - 1 <= (causal ? C - w : C - 1);   // to every row
       float acc = 0.f, acc2 = 0.f, acc3 = 0.f, acc4 = 0.f;
-      if (row0 + 128 * half < R) {                     // same for the whole warp
+      if (row0 + 64 * part < R) {                      // same for the whole warp
         groups([&](int g, float (&v)[32]) {
-          if (row0 + 128 * half + 32 * g >= R) return;   // 32 padding rows: nothing to add (same for the whole warp)
-          const float4* info = rowinfo + 128 * half + 32 * g;
+          if (row0 + 64 * part + 32 * g >= R) return;   // 32 padding rows: nothing to add (same for the whole warp)
+          const float4* info = rowinfo + 64 * part + 32 * g;
           if (all_visible) {
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
@@ -159,16 +165,16 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
         });
       }
       acc = (acc + acc2) + (acc3 + acc4);
-      // the half-1 warp hands its sums over (two buffers, by tile parity); the half-0 warp adds and
-      // stores.  pair_bar is the barrier of this tile's parity: its (n_done / 2)-th use.
+      // the warps of parts 1..3 hand their sums over (two buffers, by tile parity); the part-0 warp adds them in
+      // a fixed order and stores.  pair_bar is the barrier of this tile's parity: its (n_done / 2)-th use.
       const int slot = (n_done & 1) * 32 + (lane_row & 31);
-      if (half == 1) {
+      if (part != 0) {
         scratch[slot] = acc;
         tc::mbar_arrive(pair_bar);
       } else {
         if (pair_ok) pair_ok = mbar_wait_bounded(pair_bar, (n_done >> 1) & 1);
         if (pair_ok && j < C) {
-          const float tot = (acc + partner[slot]) * inv_R;
+          const float tot = ((acc + siblings(1)[slot]) + (siblings(2)[slot] + siblings(3)[slot])) * inv_R;
           sw[j] = row_block == 0 ? tot : sw[j] + tot;
         }
       }
@@ -192,7 +198,8 @@ __global__ void __launch_bounds__(kRowReduceWarps * 32)
   const Header* hdr = reinterpret_cast<const Header*>(cache);
   const Unit* u = unit_of(cache, hdr, false, blockIdx.y, nullptr);
   const int R = hdr->obs_window * hdr->group;
-  const int n_tiles = ((u->C + tc::kKeysPerTile - 1) / tc::kKeysPerTile + tiles_per_cta - 1) / tiles_per_cta;
+  // two partial statistics (one per half of the key tiles) for every key range of the unit
+  const int n_tiles = 2 * (((u->C + tc::kKeysPerTile - 1) / tc::kKeysPerTile + tiles_per_cta - 1) / tiles_per_cta);
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * kRowReduceWarps + (threadIdx.x >> 5);
   if (r >= R) return;

@@ -29,10 +29,10 @@ constexpr int kQBytes = 2 * kPlaneBytesQ;           // 64 KB
 constexpr int kStages = 3;
 constexpr int kLoadLag = 2;                         // key tiles in flight per CTA
 constexpr int kTmemCols = 512;                      // two accumulator buffers of 256 columns
-constexpr int kDrainWarps = 8;                      // two per lane quarter: columns 0..127 and 128..255
-constexpr int kThreads = (2 + kDrainWarps) * 32;    // warp 0 loads, warp 1 issues, warps 2..9 drain
+constexpr int kDrainWarps = 16;                     // four per lane quarter, 64 accumulator columns each
+constexpr int kThreads = (2 + kDrainWarps) * 32;    // warp 0 loads, warp 1 issues, warps 2..17 drain
 constexpr int kBarBytes = 256;
-constexpr int kScratchPerWarp = 4096;               // 32 x 32 floats a draining warp may use to reorder its output
+constexpr int kScratchPerWarp = 2048;               // 32 x 16 floats a draining warp may use to reorder its output
 constexpr int kSmemBytes =
     kQBytes + kStages * kStageBytes + kDrainWarps * kScratchPerWarp + kBarBytes + 1024;   // + slack to align to 1024
 
@@ -108,8 +108,8 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
                :
                : "memory");
 }
-// The four 32-column groups of a draining thread's 128 columns, the read of group g + 1 in flight
-// while fn(g, v) works on group g.  Whole warps call it.
+// The two 32-column groups of a draining thread's 64 columns, the read of the second in flight while
+// fn(0, v) works on the first.  Whole warps call it.
 template <class Fn>
 __device__ __forceinline__ void drain_groups(uint32_t taddr, Fn fn) {
   uint32_t ra[32], rb[32];
@@ -121,19 +121,9 @@ __device__ __forceinline__ void drain_groups(uint32_t taddr, Fn fn) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
   fn(0, v);
   tmem_ld_wait(rb);
-  tmem_ld32_issue(taddr + 64u, ra);
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rb[i]);
   fn(1, v);
-  tmem_ld_wait(ra);
-  tmem_ld32_issue(taddr + 96u, rb);
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
-  fn(2, v);
-  tmem_ld_wait(rb);
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rb[i]);
-  fn(3, v);
 }
 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -158,15 +148,15 @@ __device__ __forceinline__ uint32_t piece_offset(int row, int piece, int plane_b
 //   kKeysAsRows false: accumulator rows = query rows (two M = 128 blocks side by side, block t in
 //               columns 128 t .. 128 t + 127 = the tile's keys); true: accumulator rows = the tile's keys,
 //               columns = the 256 query rows
-//   epilogue    functor called by each of the 256 draining threads for every tile:
-//               epilogue(tile, lane 0..127, half 0..1, load, scratch, partner, pair_bar): the thread owns accumulator lane
-//               `lane`, columns 128 half .. 128 half + 127; groups(fn) calls fn(g, v) for g = 0..3 with its
-//               columns 128 half + 32 g .. + 31 in float v[32] and must be called by whole warps (or not at all);
-//               scratch is the warp's 4 KB of shared memory; partner is the scratch of the warp that owns
-//               the other column half of the same lanes, pair_bar a barrier (32 arrivals per phase;
-//               one for the even and one for the odd tiles of the CTA, so its k-th use has parity k & 1)
-//               the half-1 warp may use to hand data to the half-0 warp: the two accumulator buffers keep
-//               the warps within one tile of each other, so a phase is never met twice
+//   epilogue    functor called by each of the 512 draining threads for every tile:
+//               epilogue(tile, lane 0..127, part 0..3, groups, scratch, siblings, pair_bar): the thread owns
+//               accumulator lane `lane`, columns 64 part .. 64 part + 63; groups(fn) calls fn(g, v) for
+//               g = 0, 1 with its columns 64 part + 32 g .. + 31 in float v[32] and must be called by whole
+//               warps (or not at all); scratch is the warp's 2 KB of shared memory; siblings(p) is the
+//               scratch of the warp that owns part p of the same lanes; pair_bar is a barrier (96 arrivals per
+//               phase; one for the even and one for the odd tiles of the CTA, so its k-th use has parity
+//               k & 1) the warps of parts 1..3 may use to hand data to the part-0 warp: the two accumulator
+//               buffers keep the warps within one tile of each other, so a phase is never met twice
 // Returns false if a bounded wait ran out (the caller reports it); tensor memory is freed either way.
 // ---------------------------------------------------------------------------------------------
 template <bool kKeysAsRows, class QRowFn, class Epilogue>
@@ -212,7 +202,7 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
       mbar_init(acc_full + b, 1);
       mbar_init(acc_empty + b, kDrainWarps * 32);
     }
-    for (int q = 0; q < 8; ++q) mbar_init(pair_bar + q, 32);
+    for (int q = 0; q < 8; ++q) mbar_init(pair_bar + q, 96);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -302,18 +292,18 @@ __device__ bool scores_cta(uint8_t* smem_raw, QRowFn q_row, const __nv_bfloat16*
       __syncwarp();
     }
   } else {
-    // ---- drain: warp w owns lane quarter w % 4 (the hardware's rule) and column half (w - 2) / 4 ----
-    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    // ---- drain: warp w owns lane quarter w % 4 (the hardware's rule) and column part (w - 2) / 4 ----
+    const int quarter = warp & 3, part = (warp - 2) >> 2, slot = (warp - 2) & 3;
     const int row = quarter * 32 + lane;
     for (int i = 0; i < n_tiles; ++i) {
       const int buf = i & 1;
       if (!mbar_wait_bounded(acc_full + buf, (i >> 1) & 1)) { ok = false; break; }
       fence_after_sync();
       const uint32_t taddr =
-          tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * 256 + half * 128);
-      epilogue(tile_begin + i, row, half, [&](auto fn) { drain_groups(taddr, fn); },
+          tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * 256 + part * 64);
+      epilogue(tile_begin + i, row, part, [&](auto fn) { drain_groups(taddr, fn); },
                reinterpret_cast<float*>(scratch + (warp - 2) * kScratchPerWarp),
-               reinterpret_cast<float*>(scratch + ((warp - 2) ^ 4) * kScratchPerWarp),
+               [&](int p) { return reinterpret_cast<float*>(scratch + (p * 4 + slot) * kScratchPerWarp); },
                pair_bar + 2 * quarter + (i & 1));
       fence_before_sync();
       mbar_arrive(acc_empty + buf);
