@@ -351,6 +351,90 @@ def run_sweep(args):
                       "how": "4 independent layers launched round-robin from one CUDA graph per cell; graph time / launches"}))
 
 
+PHASES = [(0, "start"), (1, "pre-wait work issued"), (2, "dependency wait over"), (3, "query loads issued"),
+          (4, "own chunks scored, scores sent"), (5, "all scores received"), (20, "selection: histogram, barrier"),
+          (21, "selection: threshold bin found"), (22, "selection: candidates, barrier"), (23, "selection: ranked"),
+          (6, "selection done (list in shared memory)"), (7, "copies issued, lists written back"),
+          (14, "first tile landed"), (17, "first tile computed"), (18, "its stage re-armed"),
+          (19, "warp 0: second tile landed"), (8, "warp 0: tiles done"), (9, "all warps done"),
+          (16, "partials parked, barrier"), (10, "CTA partial sent to its owners"), (11, "partials received"),
+          (13, "output written")]
+
+
+def run_timeline(args):
+    """Phase timeline of the decode kernel: the profiling build of the library (same sources, -DHKV_PROFILE)
+    stamps the global nanosecond timer at the phase boundaries of every CTA; prints, for a middle layer of a
+    few-layer graph of the workload, the mean and the latest stamp of every phase, dynamic and static units apart,
+    relative to the end of the preceding layer."""
+    import ctypes
+    import torch
+    from paper_2604_05887_b200 import binding as hkv, build
+    lib = hkv.use_library(build.build_profile())
+    lib.hkv_profile_attach.argtypes = [ctypes.c_void_p, ctypes.c_longlong]
+    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    torch.cuda.set_device(0)
+    nl = args.layers if args.layers > 0 else 6
+    threads = min(os.cpu_count() or 8, 32)
+    Ls = [layer_inputs(args.workload, l, args.seed, threads) for l in range(nl)]
+    caches = [LayerCache(L) for L in Ls]
+    qs = [to_device_bf16(L.q[0]) for L in Ls]
+    outs = [c.new_out() for c in caches]
+    n_splits = [c.stats["n_splits"] for c in caches]
+
+    def step():
+        for c, q, o_ in zip(caches, qs, outs):
+            hkv.hkv_decode_attn(c.handle, q, o_)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    slots = 32
+    total = sum(n_splits)
+    buf = torch.zeros(total * slots, dtype=torch.int64, device="cuda")
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        step()
+        s.synchronize()
+        lib.hkv_profile_attach(buf.data_ptr(), total)       # the launches captured next take the regions in order
+        with torch.cuda.graph(g, stream=s):
+            step()
+        lib.hkv_profile_attach(None, 0)
+        for _ in range(3):
+            g.replay()
+        s.synchronize()
+    raw = buf.cpu().numpy().reshape(-1, slots).astype(np.uint64)
+    gt = (raw & np.uint64(0xFFFFFFFF)).astype(np.float64)          # global timer, ns (low 32 bits: 4.3 s, no wrap inside a replay)
+    clk = (raw >> np.uint64(32)).astype(np.int64)                  # SM cycle counter, low 32 bits
+    lay = max(1, nl - 2)
+    o0 = sum(n_splits[:lay])
+    sl = slice(o0, o0 + n_splits[lay])
+    blk, cb, prev = gt[sl], clk[sl], gt[o0 - n_splits[lay - 1]:o0]
+    prev_end = prev.max()
+    dyn = blk[:, 4] > 0
+    for kind, m in (("dynamic", dyn), ("static", ~dyn)):
+        b, c = blk[m], cb[m]
+        if not b.shape[0]:
+            continue
+        print(f"{kind} units: {b.shape[0]} CTAs.  us after the end of the preceding layer (global timer); SM cycles since the CTA's previous stamp")
+        last_k = None
+        for k, name in PHASES:
+            have = b[:, k] > 0
+            if not have.any():
+                continue
+            col = b[have, k]
+            line = f"  {name:34s} mean {(col.mean() - prev_end) / 1e3:7.2f}   last {(col.max() - prev_end) / 1e3:7.2f}"
+            if last_k is not None:
+                both = have & (b[:, last_k] > 0)
+                d = (c[both, k] - c[both, last_k]) % (1 << 32)
+                line += f"   cycles mean {d.mean():8.0f}  max {d.max():8.0f}"
+            print(line)
+            last_k = k
+    ticks = np.unique(gt[gt > 0])
+    print(f"layer: first CTA start {(blk[:, 0].min() - prev_end) / 1e3:.2f}, end {(blk.max() - prev_end) / 1e3:.2f} us "
+          f"after the preceding layer's end; the global timer ticks in steps of {np.diff(ticks)[:2000].min():.0f} ns")
+    hkv.use_library(None)
+
+
 def run_reference(args):
     """The reference arm of this tier is the CPU oracle, timed as it stands on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -394,6 +478,8 @@ def main():
     ap.add_argument("--sweep-quick", action="store_true", help="with --sweep: only budgets 10 % and 100 % at static fraction 0.5")
     ap.add_argument("--next-rows", action="store_true",
                     help="time hkv_classify_heads and the host-offload variant on layer 0 even in a reduced (--layers) run")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print the phase timeline of the decode kernel (profiling build of the library, --layers N layers, default 6)")
     ap.add_argument("--layers", type=int, default=0,
                     help="use only the first N layers of the workload (small case for profiler captures; "
                          "the line is then marked reduced and is not the headline number)")
@@ -403,6 +489,9 @@ def main():
         return
     if args.sweep:
         run_sweep(args)
+        return
+    if args.timeline:
+        run_timeline(args)
         return
 
     import torch

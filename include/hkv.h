@@ -100,8 +100,8 @@ typedef struct {
 
 /* Sizes of the two caller-owned device buffers, from HOST inputs only (no device work, no sync).
  * The keep-set of a static head always has min(budget, seq_len) tokens and a dynamic head always
- * loads min(n_chunks, ceil(budget / cs)) chunks (Appendix A: "determined by the per-head budget and
- * chunk size"), so no size depends on device data.
+ * loads min(n_chunks, ceil(budget / cs)) chunks (Appendix A, second paragraph: the number of chunks
+ * follows from the head's budget and the chunk size), so no size depends on device data.
  *   seq_lens  host int32 [B]        token count C_b of each sequence, 1 <= C_b <= max_seq_len
  *   head_type host uint8 [B, Hkv]   0 = static, 1 = dynamic (Section 3.1's classification result)
  *   budgets   host int32 [B, Hkv]   per-head token budget (Section 3.2's allocation result), >= 1;
@@ -185,11 +185,11 @@ hkv_status hkv_decode_attn_multi(hkv_cache* const* caches, const void* const* q,
 
 /* The two stages of hkv_decode_attn as separate calls (hkv_decode_attn = hkv_select_chunks followed
  * by hkv_attend on the same stream).  hkv_select_chunks scores every chunk of every dynamic head
- * against q and stores the top-k chunk ids in the cache (Appendix A: "identify relevant chunks by
- * computing the inner product between the query vector and chunk metadata").  hkv_attend runs the
- * attention of all heads over the static cache and the currently stored selection (Appendix A: "The
- * final attention output is then computed together with the static KV cache"); it needs one earlier
- * hkv_select_chunks (or hkv_decode_attn) if the cache has dynamic heads.  Same pointer rules. */
+ * against q and stores the top-k chunk ids in the cache (Appendix A, second paragraph: chunk relevance
+ * is the query's inner product with the chunk metadata).  hkv_attend runs the attention of all heads
+ * over the static cache and the currently stored selection (same paragraph: the output is computed
+ * over the static cache and the loaded chunks together); it needs one earlier hkv_select_chunks (or
+ * hkv_decode_attn) if the cache has dynamic heads.  Same pointer rules. */
 hkv_status hkv_select_chunks(hkv_cache* cache, const void* q, void* stream);
 hkv_status hkv_attend(hkv_cache* cache, const void* q, void* out, void* stream);
 
@@ -200,9 +200,9 @@ hkv_status hkv_attend(hkv_cache* cache, const void* q, void* out, void* stream);
 hkv_status hkv_decode_attn_host(hkv_cache* cache, const void* q_host, void* out_host, void* q_dev,
                                 void* out_dev, void* stream);
 
-/* Adds the token just generated to the compressed cache of one layer (Appendix A: the GPU KV buffer
- * is "updated" as decoding proceeds; Section 3.3: the buffer is "updated by dynamic heads during
- * decoding").  Reading taken here, the paper giving no rule: the new token's key / value row of
+/* Adds the token just generated to the compressed cache of one layer (Appendix A and Section 3.3 only
+ * say that the GPU KV buffer keeps changing while decoding proceeds).  Reading taken here, the paper
+ * giving no rule: the new token's key / value row of
  *   a static head   is appended to its condensed cache and is always retained (it is the most
  *                   recent context);
  *   a dynamic head  joins the chunked sequence: it goes to the open last chunk (or opens a new one),
@@ -333,6 +333,26 @@ hkv_status hkv_decode_cluster_capacity(int32_t group, int32_t* max_active_cluste
 hkv_status hkv_last_device_error(hkv_cache* cache, int32_t* code, int32_t* detail, void* stream);
 
 const char* hkv_status_string(hkv_status s);
+
+/* ---- development builds only: these symbols are NOT in libhkv.so ----
+ * Two further builds of the same sources exist beside the product library (build.py: build_checked,
+ * build_profile).  Neither changes what any call above computes. */
+#ifdef HKV_CHECKED
+/* Checked build (-DHKV_CHECKED, with a wait limit of a fraction of a second): the decode kernel
+ * validates every index that feeds an address (HKV_ERR_INDEX, the access is skipped).  This call
+ * launches one thread block that waits, bounded, on a barrier nothing ever arrives on: it must return
+ * by itself and leave HKV_ERR_TIMEOUT / detail 6 in the cache's error word, exactly as a lost copy
+ * would inside a decode step (Appendix A's per-step chunk load is where that could happen). */
+hkv_status hkv_selftest_wait_timeout(hkv_cache* cache, void* stream);
+/* Checked build: puts the cache's error word back to (0, 0); enqueued on `stream`. */
+hkv_status hkv_clear_device_error(hkv_cache* cache, void* stream);
+#endif
+#ifdef HKV_PROFILE
+/* Profiling build (-DHKV_PROFILE): thread 0 of every decode CTA writes the global nanosecond timer at
+ * the phase boundaries of the kernel (32 slots of 8 bytes per CTA) into `dev_buffer`, successive
+ * launches taking successive regions; launches that no longer fit are not recorded.  NULL detaches. */
+int hkv_profile_attach(void* dev_buffer, long long n_ctas);
+#endif
 
 #ifdef __cplusplus
 }

@@ -12,8 +12,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-# HKV_LIB (development aid): path of another build of the same library, e.g. one made with HKV_NVCC_FLAGS
-_LIB_PATH = os.environ.get("HKV_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhkv.so")
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhkv.so")
 
 HKV_OK = 0
 HKV_CAUSAL_WINDOW = 1
@@ -56,12 +55,12 @@ class HkvError(RuntimeError):
         super().__init__(f"{where}: {STATUS_NAMES.get(int(status), status)} ({status_string(status)})")
 
 
-def _load() -> C.CDLL:
-    if not os.path.exists(_LIB_PATH):
+def _load(path: str = _LIB_PATH) -> C.CDLL:
+    if not os.path.exists(path):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2604_05887_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2604_05887_b200.build` "
             "(or __graft_entry__.build()); there is no fallback path")
-    lib = C.CDLL(_LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32p, u8p = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_uint8)
     cfgp = C.POINTER(hkv_config)
     lib.hkv_plan.argtypes = [cfgp, i32p, u8p, i32p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
@@ -103,6 +102,15 @@ def _load() -> C.CDLL:
 
 
 lib = _load()
+
+
+def use_library(path: Optional[str] = None) -> C.CDLL:
+    """Point every wrapper of this module at another build of the same library (build.build_checked(),
+    build.build_profile()); None goes back to the product library.  Handles made by one build must be
+    used and destroyed with that build."""
+    global lib
+    lib = _load(path or _LIB_PATH)
+    return lib
 
 
 def status_string(status: int) -> str:

@@ -20,21 +20,26 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB_PATH):
+def needs_build(lib_path: str = LIB_PATH) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(lib_path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "hkv.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
-    if not force and not needs_build():
-        return LIB_PATH
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None) -> str:
+    """Compile every .cu under csrc/ into one shared library; returns its path.
+
+    extra_flags / out: a second build of the same sources beside the product library (the checked build
+    with -DHKV_CHECKED, the profiling build with -DHKV_PROFILE); such a build is always recompiled when
+    its sources are newer than it."""
+    lib_path = out or LIB_PATH
+    if not force and not needs_build(lib_path):
+        return lib_path
     cmd = [_nvcc(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB_PATH] + os.environ.get("HKV_NVCC_FLAGS", "").split() + [os.path.join(CSRC, s) for s in SOURCES]
+           "-o", lib_path] + list(extra_flags) + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -42,8 +47,21 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if verbose or r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
     if r.returncode != 0:
-        raise RuntimeError("nvcc failed building libhkv.so")
-    return LIB_PATH
+        raise RuntimeError(f"nvcc failed building {os.path.basename(lib_path)}")
+    return lib_path
+
+
+# Second builds of the same sources, kept beside the product library.
+CHECKED_LIB_PATH = os.path.join(PKG_DIR, "libhkv_checked.so")    # index validation + short wait limit + wait self-test
+PROFILE_LIB_PATH = os.path.join(PKG_DIR, "libhkv_profile.so")    # phase time stamps of the decode kernel
+
+
+def build_checked(force: bool = False) -> str:
+    return build_library(force, extra_flags=["-DHKV_CHECKED", "-DHKV_WAIT_CYCLES=400000000ll"], out=CHECKED_LIB_PATH)
+
+
+def build_profile(force: bool = False) -> str:
+    return build_library(force, extra_flags=["-DHKV_PROFILE"], out=PROFILE_LIB_PATH)
 
 
 if __name__ == "__main__":

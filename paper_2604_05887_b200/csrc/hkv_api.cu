@@ -329,12 +329,32 @@ hkv_status hkv_compress_offload(const hkv_config* cfg, const void* k, const void
                          host_mem, host_bytes, true, workspace, workspace_bytes, stream, out);
 }
 
+#ifdef HKV_CHECKED
+hkv_status hkv_selftest_wait_timeout(hkv_cache* c, void* stream) {
+  if (!c) return HKV_ERR_INVALID_ARG;
+  if (launch_selftest_wait(reinterpret_cast<int32_t*>(c->dev_base + c->hdr.err_off), static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return HKV_ERR_CUDA;
+  }
+  return HKV_OK;
+}
+hkv_status hkv_clear_device_error(hkv_cache* c, void* stream) {
+  if (!c) return HKV_ERR_INVALID_ARG;
+  if (cudaMemsetAsync(c->dev_base + c->hdr.err_off, 0, 8, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return HKV_ERR_CUDA;
+  }
+  return HKV_OK;
+}
+#endif
+
 #ifdef HKV_PROFILE
 static unsigned long long* g_prof = nullptr;
 static long long g_prof_ctas = 0, g_prof_cursor = 0;
 // Profiling build only: device buffer of kProfSlots x 8 bytes per CTA; successive decode launches
 // take successive regions of it (a launch that no longer fits is not recorded).
-extern "C" int hkv_profile_attach(void* dev_buffer, long long n_ctas) {
+int hkv_profile_attach(void* dev_buffer, long long n_ctas) {
   g_prof = static_cast<unsigned long long*>(dev_buffer);
   g_prof_ctas = n_ctas;
   g_prof_cursor = 0;

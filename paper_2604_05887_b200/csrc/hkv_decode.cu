@@ -12,13 +12,18 @@
 // under half an SM's shared memory so that two CTAs — of this launch or of two consecutive
 // launches — are resident per SM.
 //
+// A decode step is a chain of dependent stages (query -> chunk scores -> selection -> fetch -> attention
+// -> merge) and at small batch its latency, not the bytes, sets the time; the cross-CTA hand-overs
+// therefore use asynchronous remote stores that complete on the RECEIVER's mbarrier (st.async): the
+// receiver waits for exactly the bytes it needs and no cluster-wide barrier sits on the chain.
+//
 //   dynamic unit, selection:  the cluster's CTAs split the unit's chunk means between them; a warp
 //     takes up to 64 staged means and computes  S^T = M Q^T  (rows = chunks, columns = the group's
 //     query heads) on tensor cores; the chunk score is the float32 sum over the group's heads.
-//     Scores are pushed into the shared memory of every CTA of the cluster (distributed shared
-//     memory), a cluster barrier follows, and each CTA then runs the same exact selection on its
-//     own copy (a 256-bin value histogram finds the bin of the k-th score, the few scores of that
-//     bin are ranked exactly by key and index), so that every CTA knows the ascending list of
+//     Every score is sent to every CTA of the cluster (16-byte st.async, together with each warp's
+//     lower / upper bound of its scores); a CTA whose score barrier has received all bytes runs the
+//     same exact selection on its own copy (block_topk_blocked: one value histogram, exact ranking
+//     of the threshold bin, three block barriers), so that every CTA knows the ascending list of
 //     selected chunks without a round trip through global memory.  The lists later calls may ask
 //     for (scores, ids, token count) are written to global memory only after the attention's first
 //     copies have been issued.
@@ -30,22 +35,23 @@
 //     layout with movmatrix,  O^T += V^T P^T.  A CTA with a short list asks L2 for its tiles beyond
 //     the first ring-full as soon as it knows them.
 //   merge:  the warps of a CTA are combined in shared memory.  Groups up to 8: every CTA then sends
-//     each owner CTA its share of (m, l, O) into the owner's idle score area (distributed shared
-//     memory stores), one cluster barrier follows, and each owner reduces its slice of the output
+//     each owner CTA its share of (m, l, O) into the owner's idle score area (st.async crediting the
+//     owner's merge barrier), and each owner, once its bytes are in, reduces its slice of the output
 //     from its own shared memory in CTA-rank order.  Wider groups: the CTAs read each other's
-//     partials after the barrier and a second barrier keeps them alive.  Fixed order, no atomics:
-//     deterministic.
+//     partials after a cluster barrier and a second barrier keeps them alive.  Fixed order, no
+//     atomics: deterministic.
 //
 // Programmatic dependent launch.  Nothing the kernel does before griddepcontrol.wait depends on the
-// step's query or on an earlier decode launch: it reads the unit table, arms the barriers and has
-// the first ring-full of K/V rows (or chunk means) copied in.  A launch that follows another decode
-// launch on the stream may therefore start while its predecessor is still running; it reads q and
-// writes anything only after the wait.
+// step's query or on an earlier decode launch: it reads the unit table, arms the barriers, has
+// the first ring-full of K/V rows (or chunk means) copied in and asks L2 for the query's lines.  A
+// launch that follows another decode launch on the stream may therefore start while its predecessor
+// is still running; it reads q and writes anything only after the wait.
 //
 // K/V rows and chunk means live in HBM with their sixteen 16-byte pieces XOR-permuted by (row & 7),
 // which makes the ldmatrix reads of a staged tile bank-conflict free without any copy in shared
 // memory.
 #include <cstring>
+#include <mutex>
 
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
@@ -58,27 +64,33 @@ namespace {
 constexpr int kRingBytes = kDecStages * kStageBytes;                 // staging ring
 constexpr int kParkStride = kHeadDim + 4;                            // floats per parked output row
 constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp's (O, m, l)
-#ifndef HKV_DEC_WARPS
-#define HKV_DEC_WARPS 8
-#endif
 constexpr int kRecvMlOff = 6144;   // inside the score area: (m, l) of every sender and row, after the O slices
 static_assert(kMaxCluster * 8 * 8 + kRecvMlOff <= kSelSmemChunks * 4 && 8 * kHeadDim * 4 + 4 * 4 * kMaxCluster <= kRecvMlOff,
               "push-merge receive area fits the score area for groups up to 8");
 // A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
 // latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
 constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
-constexpr int kMaxWarps = HKV_DEC_WARPS;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
+constexpr int kMaxWarps = 8;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
 constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
 constexpr int kSelOff = kRingBytes;                                  // uint16 ids of the selected chunks
-constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 chunk scores
-constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers
-constexpr int kArmedOff = kBarsOff + kDecStages * 8;                 // per stage: sequence number of the tile it was last armed with
-constexpr int kTopkOff = kArmedOff + kDecStages * 4 + 8;             // scratch of the selection (never touched by bulk copies)
-constexpr int kSmemBytes = kTopkOff + kTopkScratchInts * 4;
+constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 chunk scores; later the merge's receive area
+constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers: ring stages, then scores, then merge
+constexpr int kScoreBar = kDecStages, kMergeBar = kDecStages + 1;
+constexpr int kArmedOff = kBarsOff + (kDecStages + 2) * 8;           // per stage: sequence number of the tile it was last armed with
+constexpr int kHistOff = kArmedOff + kDecStages * 4 + 8;             // selection: 256 bins
+constexpr int kBoundsOff = kHistOff + 256 * 4;                       // selection: (lower, upper) score bound of every warp of the cluster
+constexpr int kCandOff = kBoundsOff;                                 // selection: 32 candidates (key, index); the bounds are dead by then
+constexpr int kMiscOff = kBoundsOff + kMaxCluster * kMaxWarps * 8;   // selection: counters
+constexpr int kSmemBytes = kMiscOff + 96;
+// the slower selections (crowded threshold bin, more chunks than shared memory holds) keep their scratch in
+// the ring, which is idle between the scoring and the attention of a dynamic unit
+static_assert(kTopkScratchInts * 4 <= kStageBytes, "fallback selection scratch fits one ring stage");
+static_assert(kStageBytes % kRowBytes == 0, "staged rows start on 256-byte boundaries (the ldmatrix addresses rely on it)");
 static_assert(kDecCtasPerSm * (kSmemBytes + 1024) <= 233472, "two CTAs per SM");
 static_assert(part_off(kMaxWarps) + kPartBytes <= kRingBytes, "parking and the CTA partial reuse the idle ring");
-static_assert(part_off(1) % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0 && kTopkOff % 16 == 0,
+static_assert(part_off(1) % 16 == 0 && kSelOff % 16 == 0 && kScoresOff % 16 == 0 && kBarsOff % 8 == 0 && kHistOff % 16 == 0 &&
+                  kBoundsOff % 8 == 0 && kCandOff % 8 == 0,
               "alignment");
 
 __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
@@ -99,16 +111,18 @@ __device__ __forceinline__ int find_slot(const int32_t* prefix, int n, int x) {
 #define HKV_CHECK(cond, place)
 #endif
 
-// Profiling build (-DHKV_PROFILE): thread 0 of every CTA stamps the global nanosecond timer at the
-// phase boundaries of the kernel into a buffer attached with hkv_profile_attach.
+// Profiling build (-DHKV_PROFILE): thread 0 of every CTA stamps the phase boundaries of the kernel into a
+// buffer attached with hkv_profile_attach.  A stamp holds the low 32 bits of the global nanosecond timer
+// (coarse ticks, but one clock for all SMs) and, above them, the low 32 bits of the SM's cycle counter
+// (exact durations within a CTA).
 #ifdef HKV_PROFILE
-__device__ __forceinline__ unsigned long long global_ns() {
+__device__ __forceinline__ unsigned long long phase_stamp() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
+  return (static_cast<unsigned long long>(static_cast<uint32_t>(clock64())) << 32) | (t & 0xFFFFFFFFull);
 }
 #define HKV_STAMP(k) \
-  if (P.prof && threadIdx.x == 0) P.prof[static_cast<size_t>(blockIdx.x) * kProfSlots + (k)] = global_ns();
+  if (P.prof && threadIdx.x == 0) P.prof[static_cast<size_t>(blockIdx.x) * kProfSlots + (k)] = phase_stamp();
 #else
 #define HKV_STAMP(k)
 #endif
@@ -127,9 +141,6 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   const uint32_t crank = clustered ? cluster_ctarank() : 0u;
   HKV_STAMP(0)
   pdl_launch_dependents();
-  // "this CTA is running": has to be known before anybody touches its shared memory remotely
-  if (clustered) cluster_arrive();
-  bool bar_pending = clustered;   // an arrival on the cluster barrier that has not been waited for yet
 
   const int cid = blockIdx.x / csize;
   const int li = find_slot(P.unit_prefix, P.n, cid);
@@ -155,17 +166,57 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   int32_t* err = reinterpret_cast<int32_t*>(base + P.err_off[li]);
   const bool dynamic = utype != 0;
 
-  if (!dynamic && !do_attend) {   // nothing to select for a static unit
-    if (clustered) cluster_wait();
-    return;
-  }
+  // merge geometry (push merge): the output's G*128 elements are dealt to the cluster's CTAs in slices of
+  // `per`; CTA r owns elements [r * per, r * per + own_cnt(r))
+  const int total = G * kHeadDim;
+  const int per = (((total + csize - 1) / csize) + 3) & ~3;
+  // divisions by the cluster size, the slice length and the chunk size sit on the step's critical path
+  // further down: their multipliers are worked out here, before the dependency wait
+  const uint32_t csize_magic = clustered ? fastdiv_magic(static_cast<uint32_t>(csize)) : 0u;
+  const uint32_t per_magic = fastdiv_magic(static_cast<uint32_t>(per));
+  const bool cs_fast = cs > 1 && static_cast<uint64_t>(n_tok) * static_cast<uint64_t>(cs) < (1ull << 32);
+  const uint32_t cs_magic = cs > 1 ? fastdiv_magic(static_cast<uint32_t>(cs)) : 0u;
+  auto div_cs = [&](int x) { return cs_fast ? fastdiv(x, cs_magic) : x / cs; };
+  auto own_cnt = [&](int r) { return max(0, min(total, (r + 1) * per) - r * per); };
+
+  const bool identity = dynamic && k_sel >= n_chunks;          // every chunk is loaded: no list needed
+  const bool fits = n_chunks <= kSelSmemChunks;                // scores and ids fit shared memory
+  const bool scoring = dynamic && do_select;
+  // scores travel through shared memory (and the exchange between the cluster's CTAs) only when a selection
+  // needs them there; otherwise they go straight to global memory
+  const bool exchange = scoring && fits && !identity;
+  const int n_mt = (n_chunks + 15) >> 4;                       // 16-chunk groups, the unit of the exchange
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarsOff);
   volatile uint32_t* armed = reinterpret_cast<volatile uint32_t*>(smem + kArmedOff);
+  int* hist = reinterpret_cast<int*>(smem + kHistOff);
+  float2* bounds = reinterpret_cast<float2*>(smem + kBoundsOff);
+  int* misc = reinterpret_cast<int*>(smem + kMiscOff);
   if (tid == 0) {
 #pragma unroll
     for (int s = 0; s < kDecStages; ++s) { mbar_init(&bars[s], 1); armed[s] = 0u; }
+    mbar_init(&bars[kScoreBar], 1);
+    mbar_init(&bars[kMergeBar], 1);
     mbar_fence_init();
+    // what this CTA will receive from the cluster (itself included): every score of the unit plus one
+    // (lower, upper) bound per warp; later one slice of every CTA's partial output plus its (m, l) rows
+    if (clustered) {
+      if (exchange) mbar_arrive_expect_tx(&bars[kScoreBar], static_cast<uint32_t>(n_mt * 64 + csize * W * 8));
+      if (kPushMerge && do_attend) {
+        const int mine = own_cnt(static_cast<int>(crank));
+        mbar_arrive_expect_tx(&bars[kMergeBar], mine > 0 ? static_cast<uint32_t>(csize * (mine * 4 + G * 8)) : 0u);
+      }
+    }
+    misc[0] = 0;
+  }
+  if (exchange) { for (int i = tid; i < 256; i += W * 32) hist[i] = 0; }
+  // "this CTA is running and its barriers exist": has to be known before anybody touches its shared memory remotely
+  if (clustered) cluster_arrive();
+  bool bar_pending = clustered;   // an arrival on the cluster barrier that has not been waited for yet
+
+  if (!dynamic && !do_attend) {   // nothing to select for a static unit
+    if (clustered) cluster_wait();
+    return;
   }
   __syncthreads();
 
@@ -176,23 +227,20 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     if (armed[stage] != q + 1u) {
       const long long start = clock64();
       for (uint32_t it = 1; armed[stage] != q + 1u; ++it) {
-        if ((it & 255u) == 0u && clock64() - start > 2000000000ll) return false;
+        if ((it & 255u) == 0u && clock64() - start > HKV_WAIT_CYCLES) return false;
       }
     }
     return mbar_wait_bounded(&bars[stage], (q / kDecStages) & 1u);
   };
 
-  bool dead = false;    // a bounded wait ran out: stop issuing, keep every barrier
+  bool dead = false;    // a bounded wait ran out: stop issuing, keep every hand-over
   // ldmatrix lane roles: matrix index mi = lane >> 3
   const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_piece = lane >> 4;      // non-transposed A tile
   const int v_row = (lane & 7) + (lane >> 4) * 8, v_piece = (lane >> 3) & 1;      // transposed A tile
 
   float* sc_smem = reinterpret_cast<float*>(smem + kScoresOff);
   uint16_t* sel16 = reinterpret_cast<uint16_t*>(smem + kSelOff);
-  const bool identity = dynamic && k_sel >= n_chunks;          // every chunk is loaded: no list needed
-  const bool fast = n_chunks <= kSelSmemChunks;                // scores and ids fit shared memory
   const bool contiguous = !dynamic || identity;
-  const bool scoring = dynamic && do_select;
   bool sel_in_smem = false;
   uint32_t seq0 = 0;    // tiles the CTA's ring has carried in earlier phases
 
@@ -201,7 +249,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   auto setup_attn = [&](int nv) {
     n_valid = nv;
     const int n_tiles = (nv + kTile - 1) / kTile;
-    const int t_per = (n_tiles + csize - 1) / csize;
+    const int t_per = clustered ? fastdiv(n_tiles + csize - 1, csize_magic) : n_tiles;
     at_tile0 = static_cast<int>(crank) * t_per;
     at_n = max(0, min(n_tiles, at_tile0 + t_per) - at_tile0);
   };
@@ -222,7 +270,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       if (lane == 0) {
         size_t row = static_cast<size_t>(v0);
         if (one_chunk) {
-          const int ci = v0 / cs;
+          const int ci = div_cs(v0);
           const int sid = sel_at(ci);
           HKV_CHECK(sid >= 0 && sid < n_chunks, 102);
           row = static_cast<size_t>(sid) * cs + (v0 - ci * cs);
@@ -240,13 +288,13 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       return;
     }
     uint32_t* keys = reinterpret_cast<uint32_t*>(st + 2 * kTile * kRowBytes);
-    const int ci = v0 / cs + lane;                         // lane-th chunk touching this tile
+    const int ci = div_cs(v0) + lane;                      // lane-th chunk touching this tile
     const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
     if (need_keys) {
       const int v = v0 + lane;
       uint32_t key = lane & 7;
       if (v < v1) {
-        const int cj = v / cs;
+        const int cj = div_cs(v);
         key = static_cast<uint32_t>(sel_at(cj) * cs + (v - cj * cs)) & 7u;
       }
       keys[lane] = key;
@@ -276,38 +324,13 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
   };
 
-  // Tiles beyond the first ring-full cannot be staged yet, but their rows can already be pulled from
-  // HBM into L2, so that the later copies into the ring pay an L2 hit instead of an HBM round trip.
-  auto prefetch_attn = [&](int j) {   // whole warp; CTA tile j
-    const int v0 = (at_tile0 + j) * kTile;
-    const int v1 = min(v0 + kTile, n_valid);
-    if (contiguous || one_chunk) {
-      if (lane == 0) {
-        size_t row = static_cast<size_t>(v0);
-        if (one_chunk) {
-          const int ci = v0 / cs;
-          row = static_cast<size_t>(sel_at(ci)) * cs + (v0 - ci * cs);
-        }
-        const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * kRowBytes;
-        bulk_prefetch_l2(kplane + row * kRowBytes, bytes);
-        bulk_prefetch_l2(vplane + row * kRowBytes, bytes);
-      }
-      return;
-    }
-    const int ci = v0 / cs + lane;
-    const int p0 = max(v0, ci * cs), p1 = min(v1, (ci + 1) * cs);
-    if (p0 < p1) {
-      const size_t row = static_cast<size_t>(sel_at(ci)) * cs + (p0 - ci * cs);
-      const uint32_t bytes = static_cast<uint32_t>(p1 - p0) * kRowBytes;
-      bulk_prefetch_l2(kplane + row * kRowBytes, bytes);
-      bulk_prefetch_l2(vplane + row * kRowBytes, bytes);
-    }
-  };
-
   // ---- scoring phase: tiles of sc_rows chunk means, [sc_tile0, sc_tile0 + sc_n) for this CTA ----
   int sc_rows = 16, sc_tile0 = 0, sc_n = 0;
+  int wb_lo = 0, wb_hi = 0;   // this CTA's share of the score write-back
   if (scoring) {
     const int per_cta = (n_chunks + csize - 1) / csize;
+    wb_lo = static_cast<int>(crank) * per_cta;
+    wb_hi = min(n_chunks, wb_lo + per_cta);
     sc_rows = per_cta >= 4 * kScoreTile ? kScoreTile : (per_cta >= 2 * kScoreTile ? kScoreTile / 2 : 16);
     const int n_st = (n_chunks + sc_rows - 1) / sc_rows;
     const int st_per = (n_st + csize - 1) / csize;
@@ -329,6 +352,22 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
   };
 
+  // Short token lists are latency-bound: a chunk that is known to be selected while the list is still being
+  // built is requested from HBM into L2 at once, by one CTA of the cluster (nothing is requested that the step
+  // does not read).  Who asks for what is settled here, off the critical path.
+  bool early_on = false;
+  if (exchange && do_attend && !P.offload) {
+    const int my_tiles = ((k_sel * cs + kTile - 1) / kTile + csize - 1) / csize;
+    early_on = my_tiles <= kPrefetchMaxTiles && (tid % csize) == static_cast<int>(crank);
+  }
+  auto early = [&](int ci) {
+    if (!early_on) return;
+    const int rows = min(cs, C - ci * cs);
+    const size_t off = static_cast<size_t>(ci) * cs * kRowBytes;
+    bulk_prefetch_l2(kplane + off, static_cast<uint32_t>(rows) * kRowBytes);
+    bulk_prefetch_l2(vplane + off, static_cast<uint32_t>(rows) * kRowBytes);
+  };
+
   // ---- copies that do not depend on this step's query start before the dependency wait ----
   bool attn_armed = false;
   if (scoring) {
@@ -336,9 +375,13 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   } else if (!dynamic) {
     setup_attn(n_tok);
     for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
-    if (at_n <= kPrefetchMaxTiles) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
     attn_armed = true;
   }
+  const uint32_t* qg = reinterpret_cast<const uint32_t*>(P.q[li]) +
+                       (static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G) * (kHeadDim / 2);
+  // the query is written by whatever precedes this launch, so it may only be READ after the wait; asking L2
+  // for its lines reads nothing and lets the loads below meet them there
+  if (warp == W - 1 && lane * 32 < G * (kHeadDim / 2)) prefetch_l2_line(qg + lane * 32);
 
   HKV_STAMP(1)
   pdl_wait();
@@ -347,26 +390,26 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   // the group's queries as B fragments of  S^T = X Q^T  (columns >= G are zero)
   uint32_t qb[8][2 * NT];
   {
-    const uint32_t* q = reinterpret_cast<const uint32_t*>(P.q[li]) +
-                        (static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G) * (kHeadDim / 2);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int head = nt * 8 + g;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
-        qb[kk][2 * nt] = (head < G) ? __ldg(&q[head * 64 + kk * 8 + t]) : 0u;
-        qb[kk][2 * nt + 1] = (head < G) ? __ldg(&q[head * 64 + kk * 8 + 4 + t]) : 0u;
+        qb[kk][2 * nt] = (head < G) ? __ldg(&qg[head * 64 + kk * 8 + t]) : 0u;
+        qb[kk][2 * nt + 1] = (head < G) ? __ldg(&qg[head * 64 + kk * 8 + 4 + t]) : 0u;
       }
     }
   }
 
+  HKV_STAMP(3)
   // =============================================================================================
   // chunk scoring + top-k selection (dynamic units)
   // =============================================================================================
   if (scoring) {
-    if (clustered) { cluster_wait(); bar_pending = false; }   // every CTA of the cluster runs: pushes are safe
-    const uint32_t sc_addr = smem_u32(sc_smem);
-    const int n_mt = sc_rows >> 4;
+    if (clustered) { cluster_wait(); bar_pending = false; }   // every CTA of the cluster runs: remote stores are safe
+    const uint32_t sc_addr = smem_u32(sc_smem), sbar_addr = smem_u32(&bars[kScoreBar]);
+    const int n_mt_tile = sc_rows >> 4;
+    float wlo = INFINITY, whi = -INFINITY;    // bounds of the scores this warp computed (same in every lane)
 
     for (int j = warp; j < sc_n; j += W) {
       const int stage = j % kDecStages;
@@ -378,7 +421,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
         break;
       }
       const uint32_t mbase = smem_u32(smem + stage * kStageBytes);
-      for (int mt = 0; mt < n_mt; ++mt) {
+      for (int mt = 0; mt < n_mt_tile; ++mt) {
         if (mt * 16 >= nrow) break;
         float acc[2][NT][4];
 #pragma unroll
@@ -386,12 +429,14 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) acc[e][nt][0] = acc[e][nt][1] = acc[e][nt][2] = acc[e][nt][3] = 0.f;
         }
-        const uint32_t rowaddr = mbase + (mt * 16 + a_row) * kRowBytes;
+        // piece p of a row sits at p ^ key, and rows start on 256-byte boundaries: the address of piece
+        // 2 kk + a_piece is the row's address with the fixed low bits below, XOR (kk << 5)
         const uint32_t key = a_row & 7;     // tiles start at multiples of 16 chunks
+        const uint32_t rowaddr = (mbase + (mt * 16 + a_row) * kRowBytes) | ((key >> 1) << 5) | (((a_piece ^ key) & 1u) << 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           uint32_t a0, a1, a2, a3;
-          ldsm_x4(a0, a1, a2, a3, rowaddr + (((2 * kk + a_piece) ^ key) << 4));
+          ldsm_x4(a0, a1, a2, a3, rowaddr ^ (kk << 5));
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[kk & 1][nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
         }
@@ -428,45 +473,111 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
           v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
           v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
         }
-        const int c0 = r0 + mt * 16 + g, c1 = c0 + 8;
-        if (!fast) {   // too many chunks for shared memory: the selection reads the scores from global memory
-          if (t == 0 && c0 < n_chunks) gscores[c0] = v0;
-          if (t == 1 && c1 < n_chunks) gscores[c1] = v1;
-        } else {
-          for (int s = t; s < csize; s += 4) {
-            if (c0 < n_chunks) st_cluster_f32(mapa(sc_addr + c0 * 4, s), v0);
-            if (c1 < n_chunks) st_cluster_f32(mapa(sc_addr + c1 * 4, s), v1);
+        // Lanes of row group g now hold the scores of chunks g (v0) and g + 8 (v1) of this 16-chunk group.
+        // Regroup: every lane gets the four consecutive scores 4t .. 4t+3, the unit of the exchange.
+        const int cbase = r0 + mt * 16 + 4 * t;
+        float4 quad;
+        {
+          float a[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int src = (((t & 1) << 2) + i) << 2;      // a lane of row group 4 (t & 1) + i
+            const float x0 = __shfl_sync(0xffffffffu, v0, src), x1 = __shfl_sync(0xffffffffu, v1, src);
+            a[i] = (t & 2) ? x1 : x0;
+            if (cbase + i >= n_chunks) a[i] = -INFINITY;    // padding of the last group: never selected
           }
+          quad = make_float4(a[0], a[1], a[2], a[3]);
+          float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (cbase + i < n_chunks) { mn = fminf(mn, a[i]); mx = fmaxf(mx, a[i]); }
+          }
+          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          wlo = fminf(wlo, mn);
+          whi = fmaxf(whi, mx);
+        }
+        if (!exchange) {   // no selection in shared memory: the scores go to global memory
+          if (g == 0) {
+            if (cbase < n_chunks) gscores[cbase] = quad.x;
+            if (cbase + 1 < n_chunks) gscores[cbase + 1] = quad.y;
+            if (cbase + 2 < n_chunks) gscores[cbase + 2] = quad.z;
+            if (cbase + 3 < n_chunks) gscores[cbase + 3] = quad.w;
+          }
+        } else if (!clustered) {
+          if (g == 0) *reinterpret_cast<float4*>(sc_smem + cbase) = quad;
+        } else {
+          for (int s = g; s < csize; s += 8) st_async_f32x4(mapa(sc_addr + cbase * 4, s), quad, mapa(sbar_addr, s));
         }
       }
       __syncwarp();
       if (j + kDecStages < sc_n) issue_score(j + kDecStages);
     }
     seq0 = static_cast<uint32_t>(sc_n);
+    if (exchange) {
+      // this warp's bounds, to every CTA (a warp that gave up sends them too: the byte count must add up)
+      const int slot = static_cast<int>(crank) * W + warp;
+      if (!clustered) { if (lane == 0) bounds[slot] = make_float2(wlo, whi); }
+      else if (lane < csize) st_async_f32x2(mapa(smem_u32(&bounds[slot]), lane), wlo, whi, mapa(sbar_addr, lane));
+    }
     HKV_STAMP(4)
 
-    // every score of the unit is now on its way to every CTA of the cluster
-    if (!fast) __threadfence();
-    if (clustered) { cluster_arrive(); cluster_wait(); } else { __syncthreads(); }
-
-    HKV_STAMP(5)
-    int* hist = reinterpret_cast<int*>(smem + kTopkOff);
-    int* wsum = hist + 256;
-    int* bc = wsum + 96;
-    int emitted;
+    int emitted = 0;
     if (identity) {
       emitted = n_chunks;
-    } else if (fast) {
-      emitted = block_topk_smem<W>(
-          sc_smem, n_chunks, k_sel, [&](int pos, int i) { sel16[pos] = static_cast<uint16_t>(i); }, hist);
-      sel_in_smem = true;
+      __syncthreads();   // the ring turns from chunk means to K/V tiles: every warp must be done with its means
+    } else if (exchange) {
+      // every score of the unit is on its way to this CTA: wait for the bytes, not for the cluster
+      if (clustered) {
+        if (!mbar_wait_bounded_cluster(&bars[kScoreBar], 0u)) {
+          if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrExchangeWait; }
+          dead = true;
+        }
+      } else {
+        __syncthreads();
+      }
+      dead = __syncthreads_or(dead ? 1 : 0) != 0;
+      HKV_STAMP(5)
+      if (!dead) {
+        float lo = INFINITY, hi = -INFINITY;
+        for (int i = lane; i < csize * W; i += 32) { const float2 b2 = bounds[i]; lo = fminf(lo, b2.x); hi = fmaxf(hi, b2.y); }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+          hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+        }
+        uint2* cand = reinterpret_cast<uint2*>(smem + kCandOff);
+        const int ipt = (n_chunks + W * 32 - 1) / (W * 32);
+        auto stamp = [&](int k2) { HKV_STAMP(20 + k2) };
+        emitted = -1;
+        if (ipt <= 1) emitted = block_topk_blocked<W, 1>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 2) emitted = block_topk_blocked<W, 2>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 4) emitted = block_topk_blocked<W, 4>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 8) emitted = block_topk_blocked<W, 8>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        if (emitted < 0) {
+          // crowded threshold bin (or more scores than the fast path takes): the general selection, its
+          // scratch in the idle ring
+          emitted = block_topk_smem<W>(
+              sc_smem, n_chunks, k_sel, [&](int pos, int i) { sel16[pos] = static_cast<uint16_t>(i); },
+              reinterpret_cast<int*>(smem));
+          fence_proxy_async();   // the ring goes back to the bulk copies
+          __syncthreads();
+        }
+        sel_in_smem = true;
+      }
     } else {
-      // every CTA of the cluster writes the same list to the same place
+      // more chunks than shared memory holds: selection on the scores in global memory; every CTA of the
+      // cluster writes the same list to the same place
+      __threadfence();
+      if (clustered) { cluster_arrive(); cluster_wait(); } else { __syncthreads(); }
+      HKV_STAMP(5)
+      int* fb = reinterpret_cast<int*>(smem);
       emitted = block_select_emit(
           n_chunks, k_sel, [&](int i) { return float_key(__ldcg(&gscores[i])); }, [](int) { return false; },
-          [&](int pos, int i) { gsel[pos] = i; }, hist, wsum, bc);
+          [&](int pos, int i) { gsel[pos] = i; }, fb, fb + 256, fb + 256 + 96);
+      fence_proxy_async();
+      __syncthreads();
     }
-    __syncthreads();
     int nv = emitted * cs;
     if (emitted > 0) {
       const int last = identity ? n_chunks - 1 : (sel_in_smem ? static_cast<int>(sel16[emitted - 1]) : gsel[emitted - 1]);
@@ -477,23 +588,20 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     // the attention's first copies are what the step waits for: start them before anything else
     if (do_attend && !dead) {
       for (int j = warp; j < min(at_n, kDecStages); j += W) issue_attn(j);
-      if (at_n <= kPrefetchMaxTiles && !P.offload) { for (int j = kDecStages + warp; j < at_n; j += W) prefetch_attn(j); }
       attn_armed = true;
     }
     // what later calls may ask for (scores, selected ids, attended tokens), off the critical path
-    if (fast) {
-      const int c_per = (n_chunks + csize - 1) / csize;
-      const int c_end = min(n_chunks, static_cast<int>(crank + 1) * c_per);
-      for (int i = static_cast<int>(crank) * c_per + tid; i < c_end; i += W * 32) gscores[i] = sc_smem[i];
+    if (exchange && !dead) {
+      for (int i = wb_lo + tid; i < wb_hi; i += W * 32) gscores[i] = sc_smem[i];
     }
-    if (crank == 0) {
+    if (crank == 0 && !dead) {
       if (identity) { for (int i = tid; i < n_chunks; i += W * 32) gsel[i] = i; }
       else if (sel_in_smem) { for (int i = tid; i < emitted; i += W * 32) gsel[i] = sel16[i]; }
       if (tid == 0) *n_valid_g = nv;
     }
     if (!do_attend) return;
     // "my selection is done": from here on my score area is free to receive the peers' partial results
-    if (clustered && kPushMerge) { cluster_arrive_relaxed(); bar_pending = true; }
+    if (clustered && kPushMerge && !bar_pending) { cluster_arrive_relaxed(); bar_pending = true; }
   } else if (dynamic) {
     setup_attn(__ldcg(n_valid_g));   // attention only: the list of an earlier selection
   }
@@ -529,7 +637,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
 #ifdef HKV_PROFILE
     if (j == 0) { HKV_STAMP(14) }
-    if (warp == 0 && j / W < 4) { HKV_STAMP(16 + 2 * (j / W)) }
+    if (warp == 0 && j == W) { HKV_STAMP(19) }
 #endif
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(st + 2 * kTile * kRowBytes);
 #ifdef HKV_CHECKED
@@ -552,7 +660,8 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 
     // S^T = K Q^T : rows = tokens (two 16-row tiles), columns = query heads; the reduction over the
     // head dimension runs as two interleaved accumulation chains.  Piece p of a row sits at
-    // p ^ key:  (2 kk + a_piece) ^ key = ((kk ^ (key >> 1)) << 1) | ((a_piece ^ key) & 1).
+    // p ^ key:  (2 kk + a_piece) ^ key = ((kk ^ (key >> 1)) << 1) | ((a_piece ^ key) & 1); rows start on
+    // 256-byte boundaries, so that address is the row's with fixed low bits, XOR (kk << 5).
     float s[2][NT][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
@@ -564,12 +673,11 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       }
       const int r = mt * 16 + a_row;
       const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(a_row & 7);
-      const uint32_t rowaddr = kbase + r * kRowBytes + (((a_piece ^ key) & 1u) << 4);
-      const uint32_t kx = key >> 1;
+      const uint32_t rowaddr = (kbase + r * kRowBytes) | ((key >> 1) << 5) | (((a_piece ^ key) & 1u) << 4);
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
         uint32_t a0, a1, a2, a3;
-        ldsm_x4(a0, a1, a2, a3, rowaddr + ((kk ^ kx) << 5));
+        ldsm_x4(a0, a1, a2, a3, rowaddr ^ (kk << 5));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           if (kk & 1) mma_bf16(s2[nt], a0, a1, a2, a3, qb[kk][2 * nt], qb[kk][2 * nt + 1]);
@@ -638,21 +746,23 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     for (int ks = 0; ks < 2; ++ks) {
       const int r = ks * 16 + v_row;
       const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(v_row & 7);
-      const uint32_t rowaddr = vbase + r * kRowBytes + (((v_piece ^ key) & 1u) << 4);
-      const uint32_t kx = key >> 1;
+      const uint32_t rowaddr = (vbase + r * kRowBytes) | ((key >> 1) << 5) | (((v_piece ^ key) & 1u) << 4);
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
         uint32_t a0, a1, a2, a3;
-        ldsm_x4_trans(a0, a1, a2, a3, rowaddr + ((dt ^ kx) << 5));
+        ldsm_x4_trans(a0, a1, a2, a3, rowaddr ^ (dt << 5));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) mma_bf16(o[dt][nt], a0, a1, a2, a3, pb[ks][nt][0], pb[ks][nt][1]);
       }
     }
     __syncwarp();
 #ifdef HKV_PROFILE
-    if (warp == 0 && j / W < 4) { HKV_STAMP(17 + 2 * (j / W)) }
+    if (j == 0) { HKV_STAMP(17) }
 #endif
     if (j + kDecStages < at_n) issue_attn(j + kDecStages);
+#ifdef HKV_PROFILE
+    if (j == 0) { HKV_STAMP(18) }
+#endif
   }
 
   HKV_STAMP(8)
@@ -697,17 +807,16 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
   }
   __syncthreads();
+  HKV_STAMP(16)
 
   const size_t out_row0 = static_cast<size_t>(ub) * Hq + static_cast<size_t>(uh) * G;
   float* part = reinterpret_cast<float*>(smem + (W * kParkBytes));
   float2* part_ml = reinterpret_cast<float2*>(smem + (W * kParkBytes) + kMaxGroup * kHeadDim * 4);
-  // Push merge (groups up to 8): the output's G*128 elements are dealt to the cluster's CTAs in
-  // slices of `per`; every CTA sends each owner its share of (m, l, O) into the owner's score area,
-  // which is idle by now (peers have signalled the end of their selection), so that after one
-  // cluster barrier each owner reduces from its own shared memory and nobody has to wait again.
-  const int total = G * kHeadDim;
-  const int per = (((total + csize - 1) / csize) + 3) & ~3;
+  // Push merge (groups up to 8): every CTA sends each owner its share of (m, l, O) into the owner's score
+  // area, which is idle by now (peers have signalled the end of their selection), crediting the owner's
+  // merge barrier; an owner reduces from its own shared memory once its bytes are in.
   const uint32_t recv_acc = smem_u32(smem + kScoresOff), recv_ml = recv_acc + kRecvMlOff;
+  const uint32_t mbar_addr = smem_u32(&bars[kMergeBar]);
   if (clustered && kPushMerge && bar_pending) { cluster_wait(); bar_pending = false; }
   // items = (row, group of four columns): independent loads, one pass for groups up to 4, two up to 8
   for (int item = tid; item < G * 32; item += W * 32) {
@@ -724,7 +833,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #pragma unroll
       for (int w2 = 0; w2 < W; ++w2) {
         const float* po = reinterpret_cast<const float*>(smem + w2 * kParkBytes);
-        const float f = exp2f(mw[w2] - M);
+        const float f = fast_exp2(mw[w2] - M);
         const float4 v = *reinterpret_cast<const float4*>(po + row * kParkStride + dq * 4);
         acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
         L += po[16 * kParkStride + 16 + row] * f;
@@ -744,11 +853,11 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       }
     } else if (kPushMerge) {
       const int e0 = row * kHeadDim + dq * 4;
-      const int owner = e0 / per;
-      st_cluster_f32x4(mapa(recv_acc + (static_cast<int>(crank) * per + (e0 - owner * per)) * 4, owner), acc);
-      if (dq == 0) {
-        for (int s2 = 0; s2 < csize; ++s2) st_cluster_f32x2(mapa(recv_ml + (static_cast<int>(crank) * G + row) * 8, s2), M, L);
-      }
+      const int owner = fastdiv(e0, per_magic);
+      st_async_f32x4(mapa(recv_acc + (static_cast<int>(crank) * per + (e0 - owner * per)) * 4, owner), acc, mapa(mbar_addr, owner));
+      // the row's (m, l) goes to every owner: the 32 lanes of an item row hold the same pair, lane s sends to owner s
+      if (dq < csize && own_cnt(dq) > 0)
+        st_async_f32x2(mapa(recv_ml + (static_cast<int>(crank) * G + row) * 8, dq), M, L, mapa(mbar_addr, dq));
     } else {
       *reinterpret_cast<float4*>(part + row * kHeadDim + dq * 4) = acc;
       if (dq == 0) part_ml[row] = make_float2(M, L);
@@ -758,24 +867,35 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   if (!clustered) return;
 
   if (kPushMerge) {
-    cluster_arrive();
-    cluster_wait();
+    const int e_lo = static_cast<int>(crank) * per, e_hi = min(total, e_lo + per);
+    if (tid >= e_hi - e_lo) return;    // nothing of this thread's is left; peers only write to this CTA, which stays until its reducers leave
+    if (!mbar_wait_bounded_cluster(&bars[kMergeBar], 0u)) {
+      if (atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT) == 0) err[1] = kErrMergeWait;
+      return;
+    }
     HKV_STAMP(11)
     const float* racc = reinterpret_cast<const float*>(smem + kScoresOff);
     const float2* rml = reinterpret_cast<const float2*>(smem + kScoresOff + kRecvMlOff);
-    const int e_lo = static_cast<int>(crank) * per, e_hi = min(total, e_lo + per);
     for (int e = e_lo + tid; e < e_hi; e += W * 32) {
       const int row = e >> 7, le = e - e_lo;
+      // senders in two halves of eight (the second only for clusters above eight CTAs); fixed order
       float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
 #pragma unroll
-      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) { ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f; }
+#pragma unroll
+      for (int s2 = 0; s2 < 8; ++s2) {
         if (s2 < csize) {
           const float2 ml = rml[s2 * G + row];
-          ms[s2] = ml.x;
-          ls[s2] = ml.y;
-          av[s2] = racc[s2 * per + le];
-        } else {
-          ms[s2] = -INFINITY; ls[s2] = 0.f; av[s2] = 0.f;
+          ms[s2] = ml.x; ls[s2] = ml.y; av[s2] = racc[s2 * per + le];
+        }
+      }
+      if (csize > 8) {
+#pragma unroll
+        for (int s2 = 8; s2 < kMaxCluster; ++s2) {
+          if (s2 < csize) {
+            const float2 ml = rml[s2 * G + row];
+            ms[s2] = ml.x; ls[s2] = ml.y; av[s2] = racc[s2 * per + le];
+          }
         }
       }
       float M = -INFINITY;
@@ -784,19 +904,27 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
       float acc = 0.f, L = 0.f;
       if (M > -INFINITY) {
 #pragma unroll
-        for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-          const float f = exp2f(ms[s2] - M);
+        for (int s2 = 0; s2 < 8; ++s2) {
+          const float f = fast_exp2(ms[s2] - M);
           acc += av[s2] * f;
           L += ls[s2] * f;
         }
+        if (csize > 8) {
+#pragma unroll
+          for (int s2 = 8; s2 < kMaxCluster; ++s2) {
+            const float f = fast_exp2(ms[s2] - M);
+            acc += av[s2] * f;
+            L += ls[s2] * f;
+          }
+        }
       }
-      const float r = L > 0.f ? acc / L : 0.f;
+      const float r = L > 0.f ? __fdividef(acc, L) : 0.f;
       const size_t off = out_row0 * kHeadDim + e;
       if (P.out_f32) reinterpret_cast<float*>(P.out[li])[off] = r;
       else reinterpret_cast<__nv_bfloat16*>(P.out[li])[off] = __float2bfloat16_rn(r);
     }
     HKV_STAMP(13)
-    return;   // nothing of this CTA is read remotely after the barrier above
+    return;
   }
 
   // ---- merge the CTAs of the cluster through distributed shared memory ----
@@ -806,10 +934,9 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   HKV_STAMP(11)
   {
     const uint32_t part_addr = smem_u32(part), ml_addr = smem_u32(part_ml);
-    const int total = G * kHeadDim;
-    const int per = (total + csize - 1) / csize;
-    const int e_end = min(total, static_cast<int>(crank + 1) * per);
-    for (int e = static_cast<int>(crank) * per + tid; e < e_end; e += W * 32) {
+    const int per2 = (total + csize - 1) / csize;
+    const int e_end = min(total, static_cast<int>(crank + 1) * per2);
+    for (int e = static_cast<int>(crank) * per2 + tid; e < e_end; e += W * 32) {
       const int row = e >> 7;
       float ms[kMaxCluster], ls[kMaxCluster], av[kMaxCluster];
 #pragma unroll
@@ -872,18 +999,27 @@ void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int n_clust
   cfg.attrs = attr;
 }
 
-// One-time set-up of a kernel instance: shared-memory size, permission for clusters above eight
-// CTAs, and for every cluster size how many clusters the device can hold at once.
+// Once per device and kernel instance: shared-memory size, permission for clusters above eight CTAs, and
+// for every cluster size how many clusters the device can hold at once (function attributes and
+// occupancy belong to the device that is current when they are set / asked for).
 struct ClusterCaps {
   bool ready = false;
   int max_active[kMaxCluster + 1] = {};
 };
+constexpr int kMaxDevices = 64;
+std::mutex g_caps_mutex;
 
 template <int NT>
 cudaError_t configure(const ClusterCaps** out) {
-  static ClusterCaps caps;
+  static ClusterCaps caps_of[kMaxDevices];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_caps_mutex);
+  ClusterCaps& caps = caps_of[dev];
   if (!caps.ready) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<NT, warps_of(NT)>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(decode_kernel<NT, warps_of(NT)>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(decode_kernel<NT, warps_of(NT)>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
@@ -937,6 +1073,25 @@ cudaError_t decode_cluster_caps(int group, const int** max_active) {
   *max_active = caps->max_active;
   return cudaSuccess;
 }
+
+#ifdef HKV_CHECKED
+namespace {
+// Checked build only: one CTA waits, bounded, on an mbarrier that nothing ever arrives on, and records the
+// give-up in the error word like every other wait of the library does.
+__global__ void selftest_wait_kernel(int32_t* err) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  __syncthreads();
+  if (!mbar_wait_bounded(&bar, 0u)) {
+    if (threadIdx.x == 0 && atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT) == 0) err[1] = kErrSelfTest;
+  }
+}
+}  // namespace
+cudaError_t launch_selftest_wait(int32_t* err_word, cudaStream_t stream) {
+  selftest_wait_kernel<<<1, 64, 0, stream>>>(err_word);
+  return cudaGetLastError();
+}
+#endif
 
 cudaError_t launch_decode(const DecodeParams& params, int total_units, cudaStream_t stream) {
   if (total_units <= 0) return cudaSuccess;

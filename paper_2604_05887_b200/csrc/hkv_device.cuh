@@ -39,14 +39,41 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait (about a second of SM clocks): returns false when the limit ran out; the caller
-// records an error and leaves instead of spinning for ever.
+// Limit of every device-side wait, in SM clocks (about a second at full clock).
+#ifndef HKV_WAIT_CYCLES
+#define HKV_WAIT_CYCLES 2000000000ll
+#endif
+// Bounded wait: returns false when the limit ran out; the caller records an error and leaves
+// instead of spinning for ever.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long start = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u && clock64() - start > 2000000000ll) return false;
+    if ((it & 255u) == 0u && clock64() - start > HKV_WAIT_CYCLES) return false;
+  }
+}
+// The same wait with acquire semantics at cluster scope: for barriers whose bytes are delivered by
+// other CTAs of the cluster (st.async below).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long start = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((it & 255u) == 0u && clock64() - start > HKV_WAIT_CYCLES) return false;
   }
 }
 // global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16.
@@ -131,6 +158,23 @@ __device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float4 v) {
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
                : "memory");
 }
+// Asynchronous stores into the shared memory of a CTA of the cluster (addr, bar: shared::cluster addresses
+// of the SAME destination CTA, from mapa): the value is written and its byte count is credited to the
+// destination's mbarrier, whose waiters then see the data.  No cluster barrier is involved.
+__device__ __forceinline__ void st_async_f32x4(uint32_t addr, float4 v, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+               "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void st_async_f32x2(uint32_t addr, float x, float y, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr),
+               "f"(x), "f"(y), "r"(bar)
+               : "memory");
+}
+// asks L2 for the 128-byte line holding p (nothing is read into the SM, nothing to wait for)
+__device__ __forceinline__ void prefetch_l2_line(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p) : "memory");
+}
 __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
   float v;
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
@@ -141,6 +185,11 @@ __device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t addr) {
   asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
   return v;
 }
+
+// ---- division by a divisor that is fixed for the whole kernel (chunk size, cluster size): the multiplier is
+// computed once, off the critical path, and x / d becomes one multiply-high.  Exact while x * d < 2^32, d > 1.
+__device__ __forceinline__ uint32_t fastdiv_magic(uint32_t d) { return 0xFFFFFFFFu / d + 1u; }
+__device__ __forceinline__ int fastdiv(int x, uint32_t magic) { return static_cast<int>(__umulhi(static_cast<uint32_t>(x), magic)); }
 
 // ---- order-preserving key of a finite float: larger float <=> larger key; every key > 0 ----
 __device__ __forceinline__ uint32_t float_key(float f) {
@@ -381,6 +430,168 @@ __device__ int block_topk_smem(const float* scores, int n, int k, EmitFn emit, i
     before += __popc(b);
   }
   return total;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The decode step's fast path of the same selection: exact top-k over at most 256 * IPT finite float
+// scores in shared memory, three block barriers in all.  Thread t owns the IPT consecutive scores
+// [t * IPT, (t + 1) * IPT) in registers, so that the ascending output order is the thread order.
+//   1. every thread bins its scores into 256 equal-width value bins between lo and hi (lower and
+//      upper bound of the scores, known to the caller) with shared-memory atomics        -> barrier
+//   2. every warp finds, redundantly, the bin of the k-th largest score; the scores of that bin are
+//      gathered as (key, index) candidates, and each warp publishes how many of its scores lie in
+//      higher bins                                                                          -> barrier
+//   3. every warp ranks the candidates (at most 32) exactly by (key, index), which gives the
+//      threshold element and, for every warp, how many selected items precede its own; one warp scan
+//      places each selected index                                                           -> barrier
+// early(i) is called, by the thread that owns score i, for every score above the threshold bin as soon
+// as that bin is known (most of the selection, well before the list exists).  stamp(0..3) is called
+// after the first barrier, the bin search, the second barrier and the ranking (profiling builds).
+// Returns k, or -1 without having written anything when the threshold bin holds more than 32 scores
+// (many near-equal scores): the caller then runs block_topk_smem.  The decision is the same in
+// every thread.  Requires 1 <= k < n <= 256 * IPT, n_pad = n rounded up to a multiple of 16 readable
+// floats, blockDim.x = 32 * NWARPS with 256 * IPT >= n.  hist: 256 ints ZEROED by the caller, cand: 32 x (key, index), misc: 1 + NWARPS
+// ints with misc[0] ZEROED by the caller.
+// ---------------------------------------------------------------------------------------------
+template <int NWARPS, int IPT, class EarlyFn, class StampFn>
+__device__ int block_topk_blocked(const float* scores, int n, int n_pad, int k, float lo, float hi, uint16_t* out,
+                                  int* hist, uint2* cand, int* misc, EarlyFn early, StampFn stamp) {
+  static_assert(IPT == 1 || IPT == 2 || IPT == 4 || IPT == 8, "items per thread");
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int i0 = tid * IPT;
+  float v[IPT];
+  if (i0 < n_pad) {
+    if constexpr (IPT == 1) {
+      v[0] = scores[i0];
+    } else if constexpr (IPT == 2) {
+      const float2 x = *reinterpret_cast<const float2*>(scores + i0);
+      v[0] = x.x; v[1] = x.y;
+    } else {
+#pragma unroll
+      for (int q = 0; q < IPT / 4; ++q) {
+        const float4 x = *reinterpret_cast<const float4*>(scores + i0 + 4 * q);
+        v[4 * q] = x.x; v[4 * q + 1] = x.y; v[4 * q + 2] = x.z; v[4 * q + 3] = x.w;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < IPT; ++e) v[e] = 0.f;
+  }
+  const float width = hi - lo;
+  // the map score -> bin only has to be monotone, so an approximate quotient will do
+  const float scale = (width > 0.f && width < INFINITY) ? __fdividef(255.0f, width) : 0.f;
+  int bin[IPT];
+#pragma unroll
+  for (int e = 0; e < IPT; ++e) {
+    bin[e] = -1;   // not an item
+    if (i0 + e < n) {
+      bin[e] = max(0, min(255, __float2int_rd((v[e] - lo) * scale)));
+      atomicAdd(&hist[bin[e]], 1);
+    }
+  }
+  __syncthreads();
+  stamp(0);
+
+  // every warp: the highest bin b with count(bins > b) < k <= count(bins >= b)
+  int tbin, need, cnt;
+  {
+    const int4 h0 = reinterpret_cast<const int4*>(hist)[lane * 2], h1 = reinterpret_cast<const int4*>(hist)[lane * 2 + 1];
+    const int loc[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+    int tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tot += loc[j];
+    int run = tot;   // becomes the sum over lanes >= this one
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int x = __shfl_down_sync(0xffffffffu, run, off);
+      if (lane + off < 32) run += x;
+    }
+    const int above = run - tot;
+    const bool mine = above < k && k <= above + tot;
+    int my_bin = 0, my_need = 0, my_cnt = 0;
+    if (mine) {
+      int acc = above;
+#pragma unroll
+      for (int j = 7; j >= 0; --j) {
+        if (acc < k && k <= acc + loc[j]) { my_bin = lane * 8 + j; my_need = k - acc; my_cnt = loc[j]; }
+        acc += loc[j];
+      }
+    }
+    const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+    tbin = __shfl_sync(0xffffffffu, my_bin, src);
+    need = __shfl_sync(0xffffffffu, my_need, src);
+    cnt = __shfl_sync(0xffffffffu, my_cnt, src);
+  }
+  stamp(1);
+  if (cnt > 32) return -1;
+
+  int gt = 0;
+#pragma unroll
+  for (int e = 0; e < IPT; ++e) {
+    if (bin[e] > tbin) early(i0 + e);   // selected whatever the ranking below says: the caller may start on it
+    gt += bin[e] > tbin;
+    if (bin[e] == tbin) {
+      const int slot = atomicAdd(&misc[0], 1);
+      cand[slot] = make_uint2(float_key(v[e]), static_cast<uint32_t>(i0 + e));
+    }
+  }
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  if (lane == 0) misc[1 + warp] = gt;
+  __syncthreads();
+  stamp(2);
+
+  // every warp: exact rank of the candidates, lane j holding candidate j
+  const uint2 mine = lane < cnt ? cand[lane] : make_uint2(0u, 0xFFFFFFFFu);
+  int rank = 0;
+  if (cnt <= 4) {   // the usual case: a handful of scores share the threshold bin
+    for (int j = 0; j < cnt; ++j) {
+      const uint32_t ok = __shfl_sync(0xffffffffu, mine.x, j), oi = __shfl_sync(0xffffffffu, mine.y, j);
+      rank += (ok > mine.x) || (ok == mine.x && oi < mine.y);
+    }
+  } else {
+    for (int j0 = 0; j0 < cnt; j0 += 8) {   // every lane reads the same candidate: broadcast loads, eight in flight
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint2 o = cand[(j0 + j) & 31];
+        rank += (j0 + j < cnt) && ((o.x > mine.x) || (o.x == mine.x && o.y < mine.y));
+      }
+    }
+  }
+  const bool c_taken = lane < cnt && rank < need;
+  const int tsrc = __ffs(__ballot_sync(0xffffffffu, lane < cnt && rank == need - 1)) - 1;
+  const uint32_t tkey = __shfl_sync(0xffffffffu, mine.x, tsrc), tidx = __shfl_sync(0xffffffffu, mine.y, tsrc);
+  // selected items that precede this warp's: those of higher bins in lower warps, and taken candidates there
+  const int owner = static_cast<int>(mine.y / (32u * IPT));
+  int before = __popc(__ballot_sync(0xffffffffu, c_taken && owner < warp));
+  {
+    const int g = (lane < NWARPS && lane < warp) ? misc[1 + lane] : 0;
+    before += __reduce_add_sync(0xffffffffu, g);
+  }
+  stamp(3);
+  uint32_t taken = 0u;
+#pragma unroll
+  for (int e = 0; e < IPT; ++e) {
+    bool tk = bin[e] > tbin;
+    if (bin[e] == tbin) {
+      const uint32_t kv = float_key(v[e]);
+      tk = kv > tkey || (kv == tkey && static_cast<uint32_t>(i0 + e) <= tidx);
+    }
+    taken |= (tk ? 1u : 0u) << e;
+  }
+  const int c = __popc(taken);
+  int incl = c;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += x;
+  }
+  int pos = before + incl - c;
+#pragma unroll
+  for (int e = 0; e < IPT; ++e) {
+    if ((taken >> e) & 1u) out[pos++] = static_cast<uint16_t>(i0 + e);
+  }
+  __syncthreads();
+  return k;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -18,9 +18,8 @@ constexpr int kAlign = 256;
 constexpr int kMaxCluster = 16;           // CTAs that may share one (sequence, kv head) unit
 
 // decode kernel launch shape
-constexpr int kDecWarps = 4;              // consumer warps per CTA
 constexpr int kDecStages = 6;             // staging ring of a CTA (tiles in flight); two CTAs fit one SM
-constexpr int kStageBytes = kTile * kRowBytes * 2 + 128;   // K tile + V tile + row keys
+constexpr int kStageBytes = kTile * kRowBytes * 2 + 256;   // K tile + V tile + row keys; a multiple of the row size, so that every staged row starts on a 256-byte boundary
 constexpr int kScoreTile = 2 * kTile;     // most chunk means one stage holds while chunks are scored
 constexpr int kSelSmemChunks = 2048;      // chunk scores / selected ids a CTA keeps in shared memory
 
@@ -88,7 +87,7 @@ struct DecodeParams {
 constexpr int kProfSlots = 32;
 
 // device error word helpers
-enum ErrPlace : int32_t { kErrDecodeWait = 1, kErrIndex = 2, kErrScoreWait = 3 };
+enum ErrPlace : int32_t { kErrDecodeWait = 1, kErrIndex = 2, kErrScoreWait = 3, kErrExchangeWait = 4, kErrMergeWait = 5, kErrSelfTest = 6 };
 
 // Upper bound on resident CTAs per SM the decode kernel is built for.
 constexpr int kDecCtasPerSm = 2;
@@ -112,6 +111,9 @@ cudaError_t launch_build_dynamic(char* cache, const void* k, const void* v, cons
                                  int max_rows, int max_chunks, cudaStream_t stream);
 cudaError_t launch_append(char* cache, const void* k_new, const void* v_new, const Header& hdr, cudaStream_t stream);
 size_t decode_smem_bytes();
+#ifdef HKV_CHECKED
+cudaError_t launch_selftest_wait(int32_t* err_word, cudaStream_t stream);
+#endif
 
 }  // namespace hkv
 

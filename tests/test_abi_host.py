@@ -19,11 +19,37 @@ def hkv():
 
 def test_every_declared_symbol_is_exported(hkv):
     header = open(os.path.join(ROOT, "include", "hkv.h")).read()
-    declared = set(re.findall(r"\b(hkv_[a-z_]+)\s*\(", header))
+    # the development section (checked / profiling builds) is not part of the product library
+    dev = re.findall(r"#ifdef HKV_(?:CHECKED|PROFILE)\n(.*?)#endif", header, flags=re.S)
+    product = header
+    for block in dev:
+        product = product.replace(block, "")
+    declared = set(re.findall(r"\b(hkv_[a-z_]+)\s*\(", product))
     assert declared, "no declarations found"
     assert declared == set(hkv.EXPORTS)
     for name in declared:
         assert hasattr(hkv.lib, name), name
+    dev_names = set(re.findall(r"\b(hkv_[a-z_]+)\s*\(", "".join(dev)))
+    assert dev_names == {"hkv_selftest_wait_timeout", "hkv_clear_device_error", "hkv_profile_attach"}
+    for name in dev_names:
+        assert not hasattr(hkv.lib, name), f"{name} must not be in the product library"
+
+
+def test_development_builds_export_their_extra_symbols():
+    """The checked and the profiling build are the same sources with one more macro; each exports the product's
+    symbols plus its own (nothing is launched here)."""
+    import ctypes
+    from paper_2604_05887_b200 import build
+    for path, extra in ((build.build_checked(), ["hkv_selftest_wait_timeout", "hkv_clear_device_error"]),
+                        (build.build_profile(), ["hkv_profile_attach"])):
+        lib = ctypes.CDLL(path)
+        for name in list(hkv_exports()) + extra:
+            assert hasattr(lib, name), (path, name)
+
+
+def hkv_exports():
+    from paper_2604_05887_b200 import binding
+    return binding.EXPORTS
 
 
 def test_status_strings(hkv):
@@ -78,8 +104,8 @@ def test_null_pointers_are_rejected(hkv):
     assert hkv.lib.hkv_cache_destroy(None) == 0
 
 
-def test_split_plan_is_one_wave_for_bench_shape(hkv):
-    """cfg2-shaped layer: the flash-decode grid must not exceed one CTA per SM (148 without a device)."""
+def test_plan_of_bench_shape_keeps_only_the_compressed_cache(hkv):
+    """cfg2-shaped layer: cache_mem stays far below the layer's full K/V."""
     from paper_2604_05887_b200.binding import hkv_config
     import ctypes as C
     sl = [32768, 30000, 27000, 25000]
