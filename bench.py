@@ -34,23 +34,47 @@ import numpy as np  # noqa: E402
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only without MEASURED_PEAKS.json
 NOMINAL_HBM_GBS = 8000.0           # the denominator the task statement names ("~8 TB/s")
 N_LAYERS = {"cfg0": 1, "cfg1": 28, "cfg2": 28, "cfg3": 28, "cfg4": 1}
-# DRAM bytes per launch of the flash-decode kernel from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 26.85e6}   # profiles/decode_kernel_cfg2.md
+N_QUERY_SETS = 8                   # distinct seeded queries per layer, rotated step by step
+STATS_REPLAYS = 500                # per-step CUDA-event pairs behind median / min / mean
 
 
-def layer_inputs(workload: str, layer: int, seed: int, threads: int):
+def kernel_revision() -> str:
+    """Identifies the decode kernel's source: ncu counters are only quoted for the revision they were taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("hkv_decode.cu", "hkv_device.cuh", "hkv_internal.h"):
+        h.update(open(os.path.join(ROOT, "paper_2604_05887_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(workload: str):
+    """DRAM bytes per launch of the decode kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+    capture summarised in profiles/decode_kernel_traffic.txt: lines `workload revision bytes`.  None when no
+    line matches the kernel as it is now (the counters then belong to an older kernel)."""
+    path = os.path.join(ROOT, "profiles", "decode_kernel_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    rev = kernel_revision()
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 3 and not line.startswith("#") and f[0] == workload and f[1] == rev:
+            return float(f[2])
+    return None
+
+
+def layer_inputs(workload: str, layer: int, seed: int, threads: int, n_steps: int = 1):
+    """One layer of a workload with `n_steps` seeded decode queries (L.q[0 .. n_steps))."""
     import hkv_inputs as hi
     if workload == "cfg0":
-        return hi.cfg0(seed=seed, layer=layer)
+        return hi.cfg0(seed=seed, layer=layer, n_steps=n_steps)
     if workload == "cfg1":
-        return hi.cfg1(layer, seed=seed, n_steps=1, threads=threads)
+        return hi.cfg1(layer, seed=seed, n_steps=n_steps, threads=threads)
     if workload == "cfg2":
-        return hi.cfg2(layer, seed=seed, threads=threads)
+        return hi.cfg2(layer, seed=seed, n_steps=n_steps, threads=threads)
     if workload == "cfg3":
-        return hi.cfg3(layer, seed=seed, threads=threads)
+        return hi.cfg3(layer, seed=seed, n_steps=n_steps, threads=threads)
     if workload == "cfg4":
-        return hi.cfg4(0.10, 0.5, 32, seed=seed, layer=layer, threads=threads)
+        return hi.cfg4(0.10, 0.5, 32, seed=seed, layer=layer, n_steps=n_steps, threads=threads)
     raise SystemExit(f"unknown workload {workload}")
 
 
@@ -64,53 +88,67 @@ WORKLOAD_TEXT = {
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons of one GPU through NVML every few milliseconds while the timed
+    regions run (reading only)."""
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period, self.rows, self.stop, self.thread = index, period_s, [], False, None
 
     def __enter__(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
-                 str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
-        return self
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
-
-    def __exit__(self, *a):
-        if self.proc:
-            time.sleep(0.15)
-            self.proc.terminate()
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = None
             try:
-                self.proc.wait(timeout=2)
-            except Exception:
-                self.proc.kill()
-
-    def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-                for n, v in zip(names, r[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(n)
+                import torch
+                uuid = str(torch.cuda.get_device_properties(self.index).uuid)
             except Exception:
                 pass
-        if not sm:
+            self.h = None
+            if uuid:
+                for cand in (f"GPU-{uuid}", uuid):
+                    try:
+                        self.h = pynvml.nvmlDeviceGetHandleByUUID(cand)
+                        break
+                    except Exception:
+                        pass
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.thread = None
+        return self
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop:
+            try:
+                self.rows.append((nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM),
+                                  nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                                  if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons")
+                                  else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __exit__(self, *a):
+        self.stop = True
+        if self.thread:
+            self.thread.join(timeout=1)
+
+    def summary(self):
+        if not self.rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        seen = 0
+        for _, r in self.rows:
+            seen |= int(r)
+        return {"sm_mhz": statistics.median(c for c, _ in self.rows), "sm_max_mhz": float(self.max_sm),
+                "reasons": sorted(n for n, b in bits.items() if seen & b), "samples": len(self.rows),
+                "how": "NVML, every 5 ms during the timed regions"}
 
 
 def measured_peak():
@@ -234,6 +272,108 @@ def measure_offload(L, dev, launches: int = 10):
             "device_error": [code, detail]}
 
 
+class StepBench:
+    """The caches of `n_layers` layers of one workload, N_QUERY_SETS seeded queries per layer, and one CUDA graph per
+    query set holding one decode step (one hkv_decode_attn per layer, layers in sequence).  Step i replays the
+    graph of query set i % N_QUERY_SETS, so consecutive steps select different chunks."""
+
+    def __init__(self, workload: str, n_layers: int, seed: int, dev, time_compress: bool = False):
+        import torch
+        from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+        self.torch, self.workload, self.n_layers, self.dev = torch, workload, n_layers, dev
+        threads = min(os.cpu_count() or 8, 32)
+        self.caches, self.qs, self.outs, self.L0, self.comp_ms, self.kv_in_bytes0 = [], [], [], None, [], 0
+        for layer in range(n_layers):
+            L = layer_inputs(workload, layer, seed, threads, n_steps=N_QUERY_SETS)
+            k_dev, v_dev = to_device_bf16(L.k, dev), to_device_bf16(L.v, dev)
+            lc = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
+            self.caches.append(lc)
+            self.qs.append([to_device_bf16(q, dev) for q in L.q])
+            self.outs.append(lc.new_out())
+            if layer == 0:
+                self.L0 = L
+                self.kv_in_bytes0 = sum(int(c) for c in L.seq_lens) * L.n_kv_heads * 512
+                if time_compress:      # compression proper: layer 0 again, after the allocator has seen these sizes once
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    for _ in range(4):
+                        e0.record()
+                        lc2 = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
+                        e1.record()
+                        torch.cuda.synchronize()
+                        self.comp_ms.append(e0.elapsed_time(e1))
+                        lc2.close()
+            del k_dev, v_dev
+        self.stats = [c.stats for c in self.caches]
+        self.algo_bytes = sum(st["algorithmic_bytes_per_step"] for st in self.stats)
+        self.launches_per_step = sum(st["launches_per_decode"] for st in self.stats)
+        self.graphs = []
+
+    def step(self, qset: int):
+        from paper_2604_05887_b200 import binding as hkv
+        for lc, q, o_ in zip(self.caches, self.qs, self.outs):
+            hkv.hkv_decode_attn(lc.handle, q[qset], o_)
+
+    def capture(self, stream):
+        torch = self.torch
+        with torch.cuda.stream(stream):
+            for s_ in range(N_QUERY_SETS):
+                self.step(s_)
+            stream.synchronize()
+            for s_ in range(N_QUERY_SETS):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    self.step(s_)
+                self.graphs.append(g)
+            stream.synchronize()
+
+    def per_step_us(self, stream, graphs, replays: int, flush=None):
+        """One CUDA-event pair per step on the launching stream; `flush` (a buffer larger than L2) is rewritten before
+        every step when the step's working set is not itself larger than L2."""
+        torch = self.torch
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(replays)]
+        with torch.cuda.stream(stream):
+            for i in range(replays):
+                if flush is not None:
+                    flush.zero_()
+                evs[i][0].record(stream)
+                graphs[i % len(graphs)].replay()
+                evs[i][1].record(stream)
+            stream.synchronize()
+        return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+    def close(self):
+        self.graphs = []
+        for lc in self.caches:
+            lc.close()
+        self.caches = []
+
+
+def spread(us):
+    us = sorted(us)
+    return {"median": statistics.median(us), "min": us[0], "mean": sum(us) / len(us), "replays": len(us)}
+
+
+def measure_step_workload(workload: str, n_layers: int, seed: int, dev, peak: float, flush):
+    """Another step workload through the same path: per-step events, median / min / mean."""
+    import torch
+    sb = StepBench(workload, n_layers, seed, dev)
+    stream = torch.cuda.Stream(device=dev)
+    sb.capture(stream)
+    big = sb.algo_bytes > 2 * 126e6
+    sb.per_step_us(stream, sb.graphs, 24, None if big else flush)
+    sp = spread(sb.per_step_us(stream, sb.graphs, 200, None if big else flush))
+    full = N_LAYERS[workload]
+    res = {"workload": f"{workload}: {WORKLOAD_TEXT[workload]}" + (f" -- REDUCED to {n_layers} of {full} layers" if n_layers != full else ""),
+           "layers": n_layers, "us_per_step": sp, "us_per_launch_median": sp["median"] / n_layers,
+           "bytes_per_step": sb.algo_bytes, "achieved_GBps": sb.algo_bytes / sp["median"] / 1e3,
+           "frac_of_measured_peak": sb.algo_bytes / sp["median"] / 1e3 / peak,
+           "frac_of_8TBps": sb.algo_bytes / sp["median"] / 1e3 / NOMINAL_HBM_GBS,
+           "l2": "a step streams more than L2 holds" if big else "L2 flushed (512 MB rewritten) before every timed step",
+           "queries": f"{N_QUERY_SETS} seeded query sets rotated step by step"}
+    sb.close()
+    return res
+
+
 def measure_other_workload(workload: str, n_caches: int, seed: int, dev, peak: float):
     """Per-launch time of the decode kernel on another workload: `n_caches` independent one-layer
     caches (distinct seeds, together larger than L2) replayed round-robin from one CUDA graph."""
@@ -243,38 +383,40 @@ def measure_other_workload(workload: str, n_caches: int, seed: int, dev, peak: f
     threads = min(os.cpu_count() or 8, 32)
     lcs, qs, outs = [], [], []
     for i in range(n_caches):
-        L = layer_inputs(workload, i, seed, threads)
+        L = layer_inputs(workload, i, seed, threads, n_steps=4)
         lc = LayerCache(L, device=dev)
-        lcs.append(lc); qs.append(to_device_bf16(L.q[0], dev)); outs.append(lc.new_out())
+        lcs.append(lc); qs.append([to_device_bf16(q, dev) for q in L.q]); outs.append(lc.new_out())
         del L
     byt = sum(lc.stats["algorithmic_bytes_per_step"] for lc in lcs) / n_caches
     stream = torch.cuda.Stream(device=dev)
-    reps, replays = 4, 25
+    reps, replays = 4, 60
     with torch.cuda.stream(stream):
-        for _ in range(3):
+        for r in range(reps):
             for lc, q, o_ in zip(lcs, qs, outs):
-                hkv.hkv_decode_attn(lc.handle, q, o_)
+                hkv.hkv_decode_attn(lc.handle, q[r], o_)
         stream.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
-            for _ in range(reps):
+            for r in range(reps):                  # every pass over the caches uses another query set
                 for lc, q, o_ in zip(lcs, qs, outs):
-                    hkv.hkv_decode_attn(lc.handle, q, o_)
+                    hkv.hkv_decode_attn(lc.handle, q[r], o_)
         for _ in range(3):
             g.replay()
         stream.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(replays):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(replays)]
+        for a, b in evs:
+            a.record(stream)
             g.replay()
-        b.record(stream)
+            b.record(stream)
         stream.synchronize()
-    us = a.elapsed_time(b) * 1e3 / (replays * reps * n_caches)
+    per = sorted(a.elapsed_time(b) * 1e3 / (reps * n_caches) for a, b in evs)
+    us = statistics.median(per)
     gbs = byt / us / 1e3
-    res = {"workload": f"{workload}: {WORKLOAD_TEXT[workload]}", "us_per_launch": us, "bytes_per_launch": byt,
+    res = {"workload": f"{workload}: {WORKLOAD_TEXT[workload]}", "us_per_launch": us, "us_per_launch_min": per[0],
+           "bytes_per_launch": byt,
            "achieved_GBps": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_8TBps": gbs / NOMINAL_HBM_GBS,
-           "how": f"{n_caches} independent caches ({byt * n_caches / 1e6:.0f} MB together, larger than L2) launched round-robin "
-                  f"from one CUDA graph; graph time / launches"}
+           "how": f"{n_caches} independent caches ({byt * n_caches / 1e6:.0f} MB together, larger than L2) launched round-robin, "
+                  f"{reps} passes with {reps} query sets in one CUDA graph; median over {replays} graph replays / launches"}
     for lc in lcs:
         lc.close()
     return res
@@ -473,7 +615,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU time spent on the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true",
-                    help="skip the extra per-launch measurement of the single-layer 32K sweep cell (cfg4)")
+                    help="skip the other workloads (cfg4 cell, cfg1, cfg3 reduced, cfg0) and the next rows")
     ap.add_argument("--sweep", action="store_true", help="run the 100-cell single-layer sweep (cfg4) instead of the step benchmark")
     ap.add_argument("--sweep-quick", action="store_true", help="with --sweep: only budgets 10 % and 100 % at static fraction 0.5")
     ap.add_argument("--next-rows", action="store_true",
@@ -496,7 +638,7 @@ def main():
 
     import torch
     from paper_2604_05887_b200 import binding as hkv          # raises if libhkv.so is missing: no fallback
-    from paper_2604_05887_b200.layer import LayerCache, to_device_bf16
+    from paper_2604_05887_b200 import replicas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the CUDA path has no CPU fallback)")
@@ -509,191 +651,156 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    peak, peak_src = measured_peak()
 
-    # ---- build the workload: generate each layer on the host, upload, compress, keep the cache ----
+    # ---- the workload: every layer generated on the host, uploaded, compressed; caches stay resident ----
     n_layers = N_LAYERS[args.workload]
     if args.layers > 0:
         n_layers = min(n_layers, args.layers)
-    threads = min(os.cpu_count() or 8, 32)
-    caches, qs, outs, L0 = [], [], [], None
-    t_gen = t_comp = 0.0
-    kv_in_bytes = 0
-    for layer in range(n_layers):
-        t0 = time.perf_counter()
-        L = layer_inputs(args.workload, layer, args.seed + 1000 * rank, threads)   # = replicas.replica_seed(seed, rank)
-        t_gen += time.perf_counter() - t0
-        k_dev, v_dev = to_device_bf16(L.k, dev), to_device_bf16(L.v, dev)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        lc = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
-        e1.record()
-        torch.cuda.synchronize()
-        t_comp += e0.elapsed_time(e1) * 1e-3
-        kv_in_bytes += sum(int(c) for c in L.seq_lens) * L.n_kv_heads * 512
-        caches.append(lc)
-        qs.append(to_device_bf16(L.q[0], dev))
-        outs.append(lc.new_out())
-        if layer == 0:
-            L0 = L
-            # compression proper: layer 0 again, after the allocator has seen these sizes once
-            comp_ms = []
-            for _ in range(4):
-                e0.record()
-                lc2 = LayerCache(L, device=dev, k_dev=k_dev, v_dev=v_dev)
-                e1.record()
-                torch.cuda.synchronize()
-                comp_ms.append(e0.elapsed_time(e1))
-                lc2.close()
-        else:
-            del L
-        del k_dev, v_dev
-    stats = [c.stats for c in caches]
-    algo_bytes = sum(s["algorithmic_bytes_per_step"] for s in stats)
-    launches_per_step = sum(s["launches_per_decode"] for s in stats)
-    resident = sum(s["cache_bytes"] for s in stats)
-
-    def step():
-        for lc, q, o_ in zip(caches, qs, outs):
-            hkv.hkv_decode_attn(lc.handle, q, o_)
-
+    sb = StepBench(args.workload, n_layers, args.seed + 1000 * rank, dev, time_compress=True)   # = replicas.replica_seed
+    algo_bytes, L0 = sb.algo_bytes, sb.L0
+    resident = sum(st["cache_bytes"] for st in sb.stats)
+    big = algo_bytes > 2 * 126e6
+    flush = None if big else torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.Stream(device=dev)
+    sb.capture(stream)
+
     with torch.cuda.stream(stream):
-        for _ in range(3):
-            step()
-        stream.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            step()
-
-        # end-to-end variant: the step's queries start in pinned host memory, outputs end there
-        q_host = torch.stack([q.cpu() for q in qs]).pin_memory()
-        out_host = torch.empty((n_layers,) + tuple(outs[0].shape), dtype=outs[0].dtype).pin_memory()
-        q_all = torch.empty_like(q_host, device=dev)
+        # end-to-end variant: every step's queries start in pinned host memory, outputs end there
+        q_host = [torch.stack([q[s_].cpu() for q in sb.qs]).pin_memory() for s_ in range(N_QUERY_SETS)]
+        out_host = torch.empty((n_layers,) + tuple(sb.outs[0].shape), dtype=sb.outs[0].dtype).pin_memory()
+        q_all = torch.empty_like(q_host[0], device=dev)
         out_all = torch.empty_like(out_host, device=dev)
-
-        def step_e2e():
-            # the library's host-buffer entry point for a whole step: all layers' queries (pinned host) ->
-            # device in one transfer, one decode launch per layer, all outputs -> pinned host, every copy
-            # enqueued by the C-ABI call itself
-            hkv.hkv_decode_step_host([lc.handle for lc in caches], q_host, out_host, q_all, out_all)
-
-        step_e2e()
+        handles = [lc.handle for lc in sb.caches]
+        # the library's host-buffer entry point for a whole step: all layers' queries (pinned host) -> device, one
+        # decode launch per layer, all outputs -> pinned host, every copy enqueued by the C-ABI call itself
+        hkv.hkv_decode_step_host(handles, q_host[0], out_host, q_all, out_all)
         stream.synchronize()
-        graph_e2e = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph_e2e, stream=stream):
-            step_e2e()
+        graphs_e2e = []
+        for s_ in range(N_QUERY_SETS):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                hkv.hkv_decode_step_host(handles, q_host[s_], out_host, q_all, out_all)
+            graphs_e2e.append(g)
         stream.synchronize()
-
-        from paper_2604_05887_b200 import replicas
 
         def barrier():
             torch.cuda.synchronize()
             replicas.barrier()
             torch.cuda.synchronize()
 
-        def timed(g, n):
+        def timed(graphs, n):
+            """EXACTLY n steps between one CUDA-event pair on the launching stream; the slowest rank's time."""
             barrier()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            for _ in range(n):
-                g.replay()
+            for i in range(n):
+                if flush is not None:
+                    flush.zero_()
+                graphs[i % len(graphs)].replay()
             b.record(stream)
             barrier()
-            ms, _, _ = replicas.aggregate_step(a.elapsed_time(b), algo_bytes, dev)   # the slowest rank's time
+            ms, _, _ = replicas.aggregate_step(a.elapsed_time(b), algo_bytes, dev)
             return ms
 
-        for _ in range(max(args.warmup, 3)):
-            graph.replay()
+        warm = max(args.warmup, 3)
+        for i in range(warm):
+            sb.graphs[i % N_QUERY_SETS].replay()
         with ClockSampler(local) as clk:
-            ms = timed(graph, args.steps)
-        for _ in range(3):
-            graph_e2e.replay()
-        ms_e2e = timed(graph_e2e, args.steps)
+            ms = timed(sb.graphs, args.steps)
+            per_step = sb.per_step_us(stream, sb.graphs, max(STATS_REPLAYS, 100), flush)
+            for i in range(3):
+                graphs_e2e[i].replay()
+            ms_e2e = timed(graphs_e2e, args.steps)
+            per_step_e2e = sb.per_step_us(stream, graphs_e2e, 200, flush)
 
-        # ---- per-launch duration of the dominant kernel (the fused decode kernel, one launch per
-        # layer), CUDA events on its stream around every launch; the selection-only and attention-only
-        # phases of the same kernel are timed the same way for the breakdown ----
-        reps = max(3, min(20, args.steps))
-
-        def per_launch(fn):
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in range(reps * n_layers)]
-            i = 0
-            for _ in range(reps):
-                for lc, q, o_ in zip(caches, qs, outs):
-                    evs[i][0].record(stream)
-                    fn(lc, q, o_)
-                    evs[i][1].record(stream)
-                    i += 1
+        # layers-batched figure (labelled; not the metric): every layer's cache in ONE launch.  A real model's
+        # layers are sequential, so this only shows what the per-layer dependency chain costs.
+        batched = None
+        if n_layers <= 32:
+            gb = torch.cuda.CUDAGraph()
+            hkv.hkv_decode_attn_multi(handles, [q[0] for q in sb.qs], sb.outs)
             stream.synchronize()
-            ms_ = [a.elapsed_time(b) for a, b in evs[n_layers:]]        # first pass is warm-up
-            return sum(ms_) / len(ms_)
-
-        fused_ms = per_launch(lambda lc, q, o_: hkv.hkv_decode_attn(lc.handle, q, o_))
-        select_ms = per_launch(lambda lc, q, o_: hkv.hkv_select_chunks(lc.handle, q))
-        attend_ms = per_launch(lambda lc, q, o_: hkv.hkv_attend(lc.handle, q, o_))
-        code, detail = hkv.hkv_last_device_error(caches[0].handle)
+            with torch.cuda.graph(gb, stream=stream):
+                hkv.hkv_decode_attn_multi(handles, [q[0] for q in sb.qs], sb.outs)
+            batched = spread(sb.per_step_us(stream, [gb], 60, flush))
+        code, detail = hkv.hkv_last_device_error(sb.caches[0].handle)
 
     world_bytes = algo_bytes * world          # every rank runs a replica of the same size (weak scaling)
     t_step = ms * 1e-3 / args.steps
     value = world_bytes / t_step / 1e9
-    peak, peak_src = measured_peak()
-    # Launch duration of the dominant kernel = timed region (CUDA events on the launching stream
-    # around the graph replays) / launches in it: one decode_kernel per layer and nothing else, so
-    # launch gaps are charged to the kernel.  The eager per-launch event pairs below are kept for
-    # the select / attend breakdown only: with ~10 us kernels they are bounded by host enqueue time.
+    # Launch duration of the dominant kernel = timed region (CUDA events on the launching stream around the
+    # graph replays) / launches in it: one decode_kernel per layer and nothing else, so launch gaps are
+    # charged to the kernel.
     fused_avg_s = t_step / n_layers
     achieved = (algo_bytes / n_layers) / fused_avg_s / 1e9
     t_e2e = ms_e2e * 1e-3 / args.steps
-    h2d = q_host.numel() * q_host.element_size()
+    h2d = q_host[0].numel() * q_host[0].element_size()
     d2h = out_host.numel() * out_host.element_size()
+    sp = spread(per_step)
+    comp_ms = min(sb.comp_ms)
 
     line = {
         "metric": "decode_attention_achieved_hbm_GBps", "value": value, "unit": "GB/s",
-        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": t_step * 1e3,
-        "us_per_step": t_step * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "n_gpus": world, "steps": args.steps, "warmup": warm, "ms_per_step": t_step * 1e3,
+        "us_per_step": t_step * 1e6, "us_per_step_stats": sp,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}"
                    + (f" -- REDUCED to {n_layers} layers (profiling case)" if n_layers != N_LAYERS[args.workload] else ""),
                    "layers": n_layers,
                    "algorithmic_bytes_per_step": algo_bytes, "resident_cache_bytes": resident,
                    "l2": "inputs larger than L2: one step streams %.0f MB of distinct KV" % (algo_bytes / 1e6)
-                   if algo_bytes > 2 * 126e6 else "WARNING: step working set near L2 size",
+                   if big else "L2 flushed (512 MB rewritten) before every step, inside the timed region",
+                   "queries": f"{N_QUERY_SETS} seeded query sets per layer, rotated step by step (one CUDA graph per set)",
                    "launch": "CUDA graph of one hkv_decode_attn per layer, layers in sequence",
-                   "compress_GBps_of_input_kv": kv_in_bytes / t_comp / 1e9,
-                   "compress_ms_per_layer": min(comp_ms),
-                   "compress_how": "hkv_compress of layer 0 repeated 4 times, fastest (the GB/s figure beside it "
-                                   "spans every layer's first compression, device allocations included)"},
+                   "timing": f"ms_per_step: one event pair around --steps steps; us_per_step_stats: one event pair per step, "
+                             f"{len(per_step)} steps",
+                   "compress_ms_per_layer": comp_ms,
+                   "compress_GBps_of_input_kv": sb.kv_in_bytes0 / (comp_ms * 1e-3) / 1e9,
+                   "compress_how": "hkv_compress of layer 0 repeated 4 times, fastest; GB/s = that layer's full K/V bytes / that time"},
         "frac_of_measured_peak": value / world / peak, "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "decode_kernel (score + top-k + flash-decode + merge, one launch per layer)",
                      "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
-                     "avg_launch_us": fused_avg_s * 1e6, "bytes_per_launch": algo_bytes / n_layers,
+                     "avg_launch_us": fused_avg_s * 1e6, "median_launch_us": sp["median"] / n_layers,
+                     "bytes_per_launch": algo_bytes / n_layers,
                      "how": "graph step time / launches per step (CUDA events on the launching stream)",
-                     "eager_event_pairs_us": {"fused": fused_ms * 1e3, "select_only": select_ms * 1e3,
-                                              "attend_only": attend_ms * 1e3, "note": "host-enqueue bound"},
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)},
+                     "traffic": ncu_traffic(args.workload), "kernel_revision": kernel_revision(),
+                     "traffic_how": "profiles/decode_kernel_traffic.txt, the row of this kernel revision (null: no capture of this revision)"},
         "e2e": {"value": world_bytes / t_e2e / 1e9, "unit": "GB/s", "us_per_step": t_e2e * 1e6,
+                "us_per_step_stats": spread(per_step_e2e),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "how": "hkv_decode_step_host: pinned host queries of all layers -> device (first layer's ahead, the rest beside the first layers), one decode launch per layer, outputs -> pinned host in four groups beside the later layers, copies enqueued by the C-ABI call, all inside the timed graph (the per-layer host entry point hkv_decode_attn_host costs two PCIe round trips per layer: 990 us/step)"},
-        "gpu_launches": launches_per_step * args.steps,
+                "how": "hkv_decode_step_host: pinned host queries of all layers -> device (first layer's ahead, the rest beside the first layers), one decode launch per layer, outputs -> pinned host in four groups beside the later layers, copies enqueued by the C-ABI call, all inside the timed graph"},
+        "layers_batched": None if batched is None else {
+            "us_per_step": batched, "GBps": algo_bytes / batched["median"] / 1e3,
+            "frac_of_measured_peak": algo_bytes / batched["median"] / 1e3 / peak,
+            "label": "NOT the metric: all layers' caches in one hkv_decode_attn_multi launch (no layer-to-layer dependency)"},
+        "gpu_launches": sb.launches_per_step * args.steps,
         "clocks": clk.summary(),
         "device_error": [code, detail],
         "paper_context": "paper reports 7.9x KV-memory reduction and 1.52x decode speed-up (whole model, NVIDIA L40S); no attention-only number",
     }
+    stats0 = sb.stats[0]
+    sb.close()
+    del sb
+    torch.cuda.empty_cache()
 
-    if rank == 0 and world == 1 and not args.no_extra and args.layers == 0 and args.workload != "cfg4":
-        # the other 32K-token configuration: one layer, batch 16 (a kernel launch four times the size)
-        del caches, qs, outs
-        torch.cuda.empty_cache()
-        line["other_workloads"] = [measure_other_workload("cfg4", 4, args.seed + 4, dev, peak)]
+    if rank == 0 and world == 1 and not args.no_extra and args.layers == 0 and args.workload == "cfg2":
+        # the other workloads through the same path (one line carries all five)
+        fl = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        others = [measure_other_workload("cfg4", 4, args.seed + 4, dev, peak)]
+        for wl, nl in (("cfg1", 28), ("cfg3", 8), ("cfg0", 1)):
+            others.append(measure_step_workload(wl, nl, args.seed + 10, dev, peak, fl))
+            torch.cuda.empty_cache()
+        del fl
+        line["other_workloads"] = others
         line["next_rows"] = [measure_classification(L0, dev), measure_offload(L0, dev)]
     elif rank == 0 and world == 1 and args.next_rows:
         line["next_rows"] = [measure_classification(L0, dev), measure_offload(L0, dev)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt, n = oracle_decode_timing(L0, args.cpu_seconds)
-        b0 = stats[0]["algorithmic_bytes_per_step"]
+        b0 = stats0["algorithmic_bytes_per_step"]
         line["cpu_baseline"] = {"value": b0 / dt / 1e9, "unit": "GB/s", "us_per_step": dt * n_layers * 1e6,
                                 "cores": blas_threads(), "kind": "oracle",
                                 "sample": f"oracle decode_layer on layer 0 of {n_layers} ({L0.batch * L0.n_kv_heads} heads), "

@@ -70,6 +70,7 @@ static_assert(kMaxCluster * 8 * 8 + kRecvMlOff <= kSelSmemChunks * 4 && 8 * kHea
 // A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
 // latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
 constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
+
 constexpr int kMaxWarps = 8;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
 constexpr int part_off(int warps) { return warps * kParkBytes; }    // CTA partial: acc[16][128] f32, (m, l)[16]
 constexpr int kPartBytes = kMaxGroup * kHeadDim * 4 + kMaxGroup * 8;
@@ -324,25 +325,29 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
   };
 
-  // ---- scoring phase: tiles of sc_rows chunk means, [sc_tile0, sc_tile0 + sc_n) for this CTA ----
-  int sc_rows = 16, sc_tile0 = 0, sc_n = 0;
+  // ---- scoring phase: this CTA's chunk means are rows [sc_row0, sc_row1) of the unit's table, staged as
+  // sc_n pieces of up to kScoreTile rows (one ring stage, one copy, one barrier each).  The unit of work is a
+  // group of 16 rows (one tensor-core tile): when all pieces fit the ring at once, the groups are dealt to
+  // the warps one by one (several warps share a staged piece); otherwise a warp takes whole pieces and
+  // re-arms their stages.
+  int sc_row0 = 0, sc_row1 = 0, sc_n = 0;
   int wb_lo = 0, wb_hi = 0;   // this CTA's share of the score write-back
+  bool sc_fine = true;
   if (scoring) {
-    const int per_cta = (n_chunks + csize - 1) / csize;
-    wb_lo = static_cast<int>(crank) * per_cta;
-    wb_hi = min(n_chunks, wb_lo + per_cta);
-    sc_rows = per_cta >= 4 * kScoreTile ? kScoreTile : (per_cta >= 2 * kScoreTile ? kScoreTile / 2 : 16);
-    const int n_st = (n_chunks + sc_rows - 1) / sc_rows;
-    const int st_per = (n_st + csize - 1) / csize;
-    sc_tile0 = static_cast<int>(crank) * st_per;
-    sc_n = max(0, min(n_st, sc_tile0 + st_per) - sc_tile0);
+    const int mt_per = (n_mt + csize - 1) / csize;
+    sc_row0 = min(n_chunks, static_cast<int>(crank) * mt_per * 16);
+    sc_row1 = min(n_chunks, sc_row0 + mt_per * 16);
+    sc_n = (sc_row1 - sc_row0 + kScoreTile - 1) / kScoreTile;
+    sc_fine = sc_n <= kDecStages;
+    wb_lo = sc_row0;
+    wb_hi = sc_row1;
   }
-  auto issue_score = [&](int j) {
+  auto issue_score = [&](int j) {   // piece j of this CTA's chunk means into stage j % stages
     if (lane == 0) {
       const int stage = j % kDecStages;
-      const int r0 = (sc_tile0 + j) * sc_rows;
-      const uint32_t bytes = static_cast<uint32_t>(min(r0 + sc_rows, n_chunks) - r0) * kRowBytes;
-      HKV_CHECK(r0 >= 0 && r0 < n_chunks && bytes <= 2u * kTile * kRowBytes, 120);
+      const int r0 = sc_row0 + j * kScoreTile;
+      const uint32_t bytes = static_cast<uint32_t>(min(r0 + kScoreTile, sc_row1) - r0) * kRowBytes;
+      HKV_CHECK(r0 >= 0 && r0 < sc_row1 && sc_row1 <= n_chunks && bytes <= 2u * kTile * kRowBytes, 120);
 #ifdef HKV_CHECKED
       if (dead) return;
 #endif
@@ -408,21 +413,23 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
   if (scoring) {
     if (clustered) { cluster_wait(); bar_pending = false; }   // every CTA of the cluster runs: remote stores are safe
     const uint32_t sc_addr = smem_u32(sc_smem), sbar_addr = smem_u32(&bars[kScoreBar]);
-    const int n_mt_tile = sc_rows >> 4;
     float wlo = INFINITY, whi = -INFINITY;    // bounds of the scores this warp computed (same in every lane)
 
-    for (int j = warp; j < sc_n; j += W) {
-      const int stage = j % kDecStages;
-      const int r0 = (sc_tile0 + j) * sc_rows;
-      const int nrow = min(sc_rows, n_chunks - r0);
-      if (!wait_tile(stage, static_cast<uint32_t>(j))) {
+    const int mt_cnt = (sc_row1 - sc_row0 + 15) >> 4;                 // 16-row groups of this CTA
+    const int n_items = sc_fine ? mt_cnt : sc_n;
+    for (int it = warp; it < n_items; it += W) {
+      const int piece = sc_fine ? (it >> 2) : it;                       // staged piece the item reads
+      const int m_lo = sc_fine ? it : it * 4, m_hi = sc_fine ? it + 1 : min(mt_cnt, it * 4 + 4);
+      const int stage = piece % kDecStages;
+      if (!wait_tile(stage, static_cast<uint32_t>(piece))) {
         if (lane == 0) { atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT); err[1] = kErrScoreWait; }
         dead = true;
         break;
       }
       const uint32_t mbase = smem_u32(smem + stage * kStageBytes);
-      for (int mt = 0; mt < n_mt_tile; ++mt) {
-        if (mt * 16 >= nrow) break;
+      for (int m = m_lo; m < m_hi; ++m) {
+        const int mt = m & 3;                                           // group within the piece
+        const int r0 = sc_row0 + piece * kScoreTile;                    // first chunk of the piece
         float acc[2][NT][4];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
@@ -511,7 +518,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
         }
       }
       __syncwarp();
-      if (j + kDecStages < sc_n) issue_score(j + kDecStages);
+      if (!sc_fine && it + kDecStages < sc_n) issue_score(it + kDecStages);
     }
     seq0 = static_cast<uint32_t>(sc_n);
     if (exchange) {

@@ -1,10 +1,12 @@
 """Comparison of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
 
 Index sets must be equal; an element may only be swapped for one whose ORACLE float32 score is tied
-with it: |s_a - s_b| < 1e-5 * max(|s_a|, |s_b|), or < 1e-5 * max|s| of that head (the second form
-covers thresholds that sit near score zero, where a purely relative test is ill-conditioned under a
-different float32 summation order).  Where sets differ by permitted swaps, outputs are compared with
-the oracle re-run on the GPU's index set.  Outputs: max-abs <= 2e-2 and mean-abs <= 2e-3.
+with it: |s_a - s_b| < 1e-5 * max(|s_a|, |s_b|).  A wider form, < 1e-5 * max|s| over the candidates
+that are actually ranked (it covers thresholds near score zero, where a purely relative test is
+ill-conditioned under a different float32 summation order), is accepted too but counted apart
+("swaps_wide"): the tests of the five workloads assert that it was never needed.  Where sets differ by
+permitted swaps, outputs are compared with the oracle re-run on the GPU's index set.  Outputs: max-abs
+<= 2e-2 and mean-abs <= 2e-3.
 """
 from __future__ import annotations
 
@@ -19,21 +21,39 @@ MAX_ABS, MEAN_ABS = 2e-2, 2e-3
 TIE_REL = 1e-5
 
 
-def sets_match_up_to_ties(gpu_ids, ref_ids, scores_f32, what=""):
-    """True if equal; if different, every swapped pair must be a score tie. Returns #swaps."""
+def sets_match_up_to_ties(gpu_ids, ref_ids, scores_f32, what="", ranked=None):
+    """Equal sets pass.  Otherwise every element the GPU took instead of one of the oracle's must be tied with
+    it in the ORACLE's float32 scores.  Returns (swaps, wide): `swaps` = elements exchanged; `wide` = those of
+    them that are ties only in the wide form, |s_a - s_b| < 1e-5 * max|s| over the RANKED candidates (`ranked`:
+    their indices; default all), not in the strict relative form |s_a - s_b| < 1e-5 * max(|s_a|, |s_b|)."""
     g, r = set(int(x) for x in gpu_ids), set(int(x) for x in ref_ids)
     assert len(g) == len(gpu_ids), f"{what}: duplicate ids from the GPU"
     assert len(g) == len(r), f"{what}: {len(g)} ids from the GPU, {len(r)} from the oracle"
     if g == r:
-        return 0
+        return 0, 0
     only_g = sorted(g - r, key=lambda i: -float(scores_f32[i]))
     only_r = sorted(r - g, key=lambda i: -float(scores_f32[i]))
-    smax = float(np.abs(scores_f32).max())
+    pool = np.asarray(scores_f32)[np.asarray(ranked, dtype=np.int64)] if ranked is not None else np.asarray(scores_f32)
+    smax = float(np.abs(pool).max()) if pool.size else 0.0
+    wide = 0
     for a, b in zip(only_g, only_r):
         sa, sb = float(scores_f32[a]), float(scores_f32[b])
-        tol = TIE_REL * max(max(abs(sa), abs(sb)), smax)
-        assert abs(sa - sb) < tol, f"{what}: GPU kept {a} (score {sa}) instead of {b} (score {sb}): not a tie"
-    return len(only_g)
+        strict = abs(sa - sb) < TIE_REL * max(abs(sa), abs(sb))
+        if not strict:
+            assert abs(sa - sb) < TIE_REL * smax, f"{what}: GPU kept {a} (score {sa}) instead of {b} (score {sb}): not a tie"
+            wide += 1
+    return len(only_g), wide
+
+
+def ranked_static_candidates(is_text_row, C, w, budget):
+    """Positions whose window score takes part in a static head's ranking: the visual tokens before the window,
+    or, when window + text do not fit the budget, the text tokens before it (none when budget <= w)."""
+    budget = int(min(budget, C))
+    if budget <= w:
+        return np.zeros(0, dtype=np.int64)
+    hist = np.arange(0, C - w, dtype=np.int64)
+    txt = hist[np.asarray(is_text_row[:C - w]) != 0]
+    return txt if txt.size >= budget - w else hist[np.asarray(is_text_row[:C - w]) == 0]
 
 
 def check_outputs(gpu_out, ref_out, what=""):
@@ -56,7 +76,7 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
     units = all_units if units is None else units
     oc = o.compress_layer(L, token_scores=token_scores, causal_window=causal, only=units,
                           scale=softmax_scale or None)
-    rep = {"swaps_static": 0, "swaps_dynamic": 0, "max_abs": 0.0, "mean_abs": 0.0, "sw_rel": 0.0}
+    rep = {"swaps_static": 0, "swaps_dynamic": 0, "swaps_wide": 0, "max_abs": 0.0, "mean_abs": 0.0, "sw_rel": 0.0}
     keep_override = {}
     for (b, h) in units:
         hd = oc.heads[(b, h)]
@@ -71,8 +91,10 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
                 rep["sw_rel"] = max(rep["sw_rel"], float(rel))
                 assert rel < 2e-5, f"s_w ({b},{h}): max error {rel:.2e} of the largest score"
                 assert abs(float(sw.astype(np.float64).sum()) - 1.0) < 1e-4
-            n = sets_match_up_to_ties(gi, hd.keep, hd.scores, f"static ({b},{h})")
+            n, wide = sets_match_up_to_ties(gi, hd.keep, hd.scores, f"static ({b},{h})",
+                                            ranked=ranked_static_candidates(L.is_text[b], hd.C, L.obs_window, L.budgets[b, h]))
             rep["swaps_static"] += n
+            rep["swaps_wide"] += wide
             if n:
                 keep_override[(b, h)] = np.sort(gi.astype(np.int64))
         else:
@@ -97,8 +119,9 @@ def compare_layer(L, flags=hkv.HKV_OUT_F32, token_scores=None, units=None, steps
                 gsc = hkv.hkv_get_chunk_scores(lc.handle, b, h, hd.summaries.shape[0])
                 smax = float(np.abs(ref_scores[(b, h)]).max()) + 1e-30
                 assert np.abs(gsc - ref_scores[(b, h)]).max() / smax < 1e-5, f"chunk scores ({b},{h})"
-            n = sets_match_up_to_ties(gsel, ref_sel[(b, h)], ref_scores[(b, h)], f"dynamic ({b},{h})")
+            n, wide = sets_match_up_to_ties(gsel, ref_sel[(b, h)], ref_scores[(b, h)], f"dynamic ({b},{h})")
             rep["swaps_dynamic"] += n
+            rep["swaps_wide"] += wide
             if n:
                 chunk_override[(b, h)] = gsel
         ref_out, _, _ = o.decode_layer(L, oc, q_bits, chunk_override=chunk_override or None,

@@ -70,7 +70,7 @@ def test_append_matches_oracle_step_by_step(cs, C, budget, cap, offload):
             else:
                 assert np.array_equal(hkv.hkv_get_summaries(lc.handle, b, h, hd.summaries.shape[0]), hd.summaries)
                 gsel = hkv.hkv_get_selected_chunks(lc.handle, b, h)
-                if P.sets_match_up_to_ties(gsel, ref_sel[(b, h)], ref_scores[(b, h)], f"step {t} ({b},{h})"):
+                if P.sets_match_up_to_ties(gsel, ref_sel[(b, h)], ref_scores[(b, h)], f"step {t} ({b},{h})")[0]:
                     override[(b, h)] = gsel
         ref_out, _, _ = o.decode_layer(L, oc, q_bits, chunk_override=override or None)
         P.check_outputs(out.cpu().numpy(), ref_out, f"after {t + 1} appended tokens")
