@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
@@ -70,7 +71,7 @@ __global__ void __launch_bounds__(kNoAllocThreads)
 
 // Device address of the scratch on each device, resolved once per device (host code cannot use the
 // array's name as a pointer: on the host it is only a handle for the runtime's symbol table).
-float* g_scratch_addr[kMaxDevices] = {};
+std::atomic<float*> g_scratch_addr[kMaxDevices];   // zero-initialised; host threads may race to fill an entry with the same value
 
 }  // namespace
 }  // namespace hkv
@@ -85,17 +86,17 @@ extern "C" hkv_status hkv_topk_chunks_noalloc(const void* q, const void* means, 
   if ((reinterpret_cast<uintptr_t>(means) & 15) || (reinterpret_cast<uintptr_t>(q) & 1)) return HKV_ERR_INVALID_ARG;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return HKV_ERR_CUDA; }
-  if (!g_scratch_addr[dev]) {
-    float* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scores) != cudaSuccess || !p) {
+  float* scratch = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&scratch), g_noalloc_scores) != cudaSuccess || !scratch) {
       cudaGetLastError();
       return HKV_ERR_CUDA;
     }
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(scratch, std::memory_order_release);
   }
   topk_chunks_kernel<<<1, kNoAllocThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(q), static_cast<const uint4*>(means), group, n_chunks, std::min(k, n_chunks),
-      g_scratch_addr[dev], out_ids);
+      scratch, out_ids);
   if (cudaGetLastError() != cudaSuccess) return HKV_ERR_CUDA;
   return HKV_OK;
 }

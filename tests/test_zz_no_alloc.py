@@ -5,17 +5,20 @@ runtime's callback, or in a loop whose latency budget rules out cudaMalloc and a
 may call it.  For them the entry point keeps its per-chunk score scratch in a fixed array inside
 the library; they hand over inputs and the output buffer only.
 
-The test drives the entry point through the C ABI twice in a row (the second call reuses the
-scratch the first one left behind, with a different query and a different chunk count) and checks
+The first test drives the entry point through the C ABI several times in a row (every call reuses the
+scratch the one before left behind, with a different query and a different chunk count) and checks
 each result against what the regular path (hkv_decode_attn -> hkv_get_selected_chunks) selects for
-the same head, under the same rule the other parity tests use: equal sets, except for swaps between
-chunks whose scores are tied to 1e-5.  It is collected last on purpose.
+the same head AND against the CPU oracle's selection from its own scores, under the rule the other
+parity tests use: equal sets, except for swaps between chunks whose oracle scores are tied to 1e-5.
+The second covers the ends of the size range against the oracle: as many chunk means as the built-in
+scratch holds, and k at or beyond the number of chunks.  The file is collected last on purpose.
 """
 import numpy as np
 import pytest
 import torch
 
 import hkv_inputs as hi
+from oracle import hkv_oracle as o
 
 pytestmark = pytest.mark.gpu
 
@@ -59,9 +62,41 @@ def test_no_alloc_selection_matches_regular_path_twice_in_a_row():
             torch.cuda.synchronize()
             got = out_ids.cpu().numpy()
             assert np.all(np.diff(got) > 0), "ids must come out ascending"
-            P.sets_match_up_to_ties(got, sel, scores, f"no-alloc ({b},{h})")
+            P.sets_match_up_to_ties(got, sel, scores, f"no-alloc vs regular path ({b},{h})")
+            ref_scores = o.chunk_scores(L.q[0][b, h * G:(h + 1) * G], means)
+            _, wide = P.sets_match_up_to_ties(got, o.select_chunks(ref_scores, sel.size), ref_scores,
+                                              f"no-alloc vs oracle ({b},{h})")
+            assert wide == 0
             n_calls += 1
     assert n_calls >= 2
+
+
+def test_no_alloc_at_the_ends_of_its_size_range():
+    """HKV_NOALLOC_MAX_CHUNKS chunk means (16 MB; the radix selection then makes several passes over the whole
+    scratch), twice in a row with different k, and k >= n_chunks (every id, in order)."""
+    from paper_2604_05887_b200 import binding as hkv
+    from paper_2604_05887_b200.layer import to_device_bf16
+    import parity_util as P
+    rng = np.random.default_rng(77)
+    G, n = 7, hkv.HKV_NOALLOC_MAX_CHUNKS
+    q = hi.f32_to_bf16_bits(rng.standard_normal((G, 128)).astype(np.float32))
+    means = hi.f32_to_bf16_bits(rng.standard_normal((n, 128)).astype(np.float32))
+    means[1000:1040] = means[1000]                      # a run of exactly equal scores: the lower ids must win
+    q_dev, means_dev = to_device_bf16(q), to_device_bf16(means)
+    ref_scores = o.chunk_scores(q, means)
+    for k in (6554, 100):
+        out_ids = torch.full((k,), -1, dtype=torch.int32, device="cuda")
+        hkv.hkv_topk_chunks_noalloc(q_dev, means_dev, k, out_ids)
+        torch.cuda.synchronize()
+        got = out_ids.cpu().numpy()
+        assert np.all(np.diff(got) > 0)
+        _, wide = P.sets_match_up_to_ties(got, o.select_chunks(ref_scores, k), ref_scores, f"no-alloc n={n} k={k}")
+        assert wide == 0
+    for n_small, k in ((37, 37), (37, 1000)):
+        out_ids = torch.full((n_small,), -1, dtype=torch.int32, device="cuda")
+        hkv.hkv_topk_chunks_noalloc(q_dev, means_dev[:n_small].contiguous(), k, out_ids)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_ids.cpu().numpy(), np.arange(n_small))
 
 
 def test_no_alloc_rejects_sizes_beyond_its_scratch():
