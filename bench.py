@@ -708,7 +708,7 @@ def main():
             sb.graphs[i % N_QUERY_SETS].replay()
         with ClockSampler(local) as clk:
             ms = timed(sb.graphs, args.steps)
-            per_step = sb.per_step_us(stream, sb.graphs, max(STATS_REPLAYS, 100), flush)
+            per_step = sb.per_step_us(stream, sb.graphs, 100 if args.layers > 0 else STATS_REPLAYS, flush)
             for i in range(3):
                 graphs_e2e[i].replay()
             ms_e2e = timed(graphs_e2e, args.steps)

@@ -384,6 +384,9 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
     P.out[i] = do_attend ? out[i] : nullptr;
     P.n_valid_off[i] = H.n_valid_off;
     P.err_off[i] = H.err_off;
+    P.dyn_list_off[i] = H.dyn_list_off;
+    P.sta_list_off[i] = H.sta_list_off;
+    P.n_dynamic[i] = H.n_dynamic;
     P.unit_prefix[i + 1] = P.unit_prefix[i] + H.n_units;
     max_tiles = std::max(max_tiles, c->max_tiles);
     n_dynamic += H.n_dynamic;
@@ -400,6 +403,17 @@ static hkv_status decode_stages(hkv_cache* const* caches, const void* const* q, 
   if (decode_cluster_caps(P.group, &max_active) != cudaSuccess) { cudaGetLastError(); return HKV_ERR_CUDA; }
   const int total_units = P.unit_prefix[n];
   P.cluster = choose_cluster(total_units, max_tiles, max_active);
+  // A launch that follows another decode launch starts, in block order, as many blocks as the device has room
+  // for beside its predecessor's.  When that is not all of them, the static units go first if they all fit:
+  // they use the head start to stage their first K/V tiles, which is worth most.  Otherwise (everything fits,
+  // or not even the static units do) the dynamic units go first: their chain of dependent stages is the
+  // longer one and must not also wait for a slot.
+  {
+    const long long slots = static_cast<long long>(max_active[P.cluster]) * P.cluster;
+    const long long all = static_cast<long long>(total_units) * P.cluster;
+    const long long sta = static_cast<long long>(total_units - n_dynamic) * P.cluster;
+    P.static_first = (2 * all > slots && sta <= slots - all) ? 1u : 0u;
+  }
   // The launch may overlap the tail of a preceding decode launch (it touches nothing that depends on
   // earlier work before its dependency wait).  Right after hkv_compress the cache itself is what
   // the preceding kernels are still writing, so that first launch is fully serialised.

@@ -145,8 +145,18 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 
   const int cid = blockIdx.x / csize;
   const int li = find_slot(P.unit_prefix, P.n, cid);
-  const int uid = cid - P.unit_prefix[li];
   char* base = P.cache[li];
+  int uid;
+  {
+    // Blocks start in index order, and a launch that follows another decode launch starts as many of them as the
+    // device has room for while its predecessor still runs: the unit type that gains most from that early
+    // start (see decode_stages) takes the cache's first clusters.
+    const int c = cid - P.unit_prefix[li], nd = P.n_dynamic[li], ns = P.unit_prefix[li + 1] - P.unit_prefix[li] - nd;
+    const int32_t* dl = reinterpret_cast<const int32_t*>(base + P.dyn_list_off[li]);
+    const int32_t* sl = reinterpret_cast<const int32_t*>(base + P.sta_list_off[li]);
+    if (P.static_first) uid = c < ns ? sl[c] : dl[c - ns];
+    else uid = c < nd ? dl[c] : sl[c - nd];
+  }
   const Unit* up = reinterpret_cast<const Unit*>(base + kUnitsOff) + uid;
   const int G = P.group, Hq = P.n_q_heads, cs = P.chunk_size;
   const int ub = uid / P.n_kv_heads, uh = uid - ub * P.n_kv_heads;

@@ -80,6 +80,10 @@ struct DecodeParams {
   void* out[kMaxMulti];
   int64_t n_valid_off[kMaxMulti];
   int64_t err_off[kMaxMulti];
+  int64_t dyn_list_off[kMaxMulti];   // unit ids of each cache's dynamic / static units: a cache's clusters take one
+  int64_t sta_list_off[kMaxMulti];   // type first, then the other (static_first)
+  int32_t n_dynamic[kMaxMulti];
+  uint32_t static_first;
 #ifdef HKV_PROFILE
   unsigned long long* prof;   // kProfSlots time stamps (ns) per CTA, or null
 #endif
