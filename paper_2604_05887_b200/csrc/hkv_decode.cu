@@ -52,6 +52,7 @@
 // memory.
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "hkv_device.cuh"
 #include "hkv_internal.h"
@@ -642,6 +643,10 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) { mrun[nt][0] = mrun[nt][1] = -INFINITY; lrun[nt][0] = lrun[nt][1] = 0.f; }
 
+  // the loop over this warp's tiles, compiled twice: rows whose 16-byte pieces follow the staged row index (the
+  // usual case: the permutation key is then a per-thread constant) and rows that carry their own keys
+  auto run_tiles = [&](auto keys_c) {
+  constexpr bool KEYS = decltype(keys_c)::value;
   for (int j = warp; j < at_n && !dead; j += W) {
     const int stage = (seq0 + j) % kDecStages;
     uint8_t* st = smem + stage * kStageBytes;
@@ -658,7 +663,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #endif
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(st + 2 * kTile * kRowBytes);
 #ifdef HKV_CHECKED
-    HKV_CHECK(!need_keys || keys[lane] < 8u, 110);
+    HKV_CHECK(!KEYS || keys[lane] < 8u, 110);
     HKV_CHECK(nrow >= 1, 111);
     dead = __any_sync(0xffffffffu, dead);
     if (dead) break;
@@ -689,7 +694,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
         s2[nt][0] = s2[nt][1] = s2[nt][2] = s2[nt][3] = 0.f;
       }
       const int r = mt * 16 + a_row;
-      const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(a_row & 7);
+      const uint32_t key = KEYS ? keys[r] : static_cast<uint32_t>(a_row & 7);
       const uint32_t rowaddr = (kbase + r * kRowBytes) | ((key >> 1) << 5) | (((a_piece ^ key) & 1u) << 4);
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
@@ -762,7 +767,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks) {
       const int r = ks * 16 + v_row;
-      const uint32_t key = need_keys ? keys[r] : static_cast<uint32_t>(v_row & 7);
+      const uint32_t key = KEYS ? keys[r] : static_cast<uint32_t>(v_row & 7);
       const uint32_t rowaddr = (vbase + r * kRowBytes) | ((key >> 1) << 5) | (((v_piece ^ key) & 1u) << 4);
 #pragma unroll
       for (int dt = 0; dt < 8; ++dt) {
@@ -781,6 +786,9 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     if (j == 0) { HKV_STAMP(18) }
 #endif
   }
+
+  };
+  if (need_keys) run_tiles(std::true_type{}); else run_tiles(std::false_type{});
 
   HKV_STAMP(8)
   // a warp that gave up tells the others, so that nobody parks results over copies still in flight
