@@ -39,11 +39,16 @@ STATS_REPLAYS = 500                # per-step CUDA-event pairs behind median / m
 
 
 def kernel_revision() -> str:
-    """Identifies the decode kernel's source: ncu counters are only quoted for the revision they were taken on."""
+    """Identifies the decode kernel's code (comments and blank space do not count): ncu counters are only quoted
+    for the revision they were taken on."""
     import hashlib
+    import re
     h = hashlib.sha256()
     for f in ("hkv_decode.cu", "hkv_device.cuh", "hkv_internal.h"):
-        h.update(open(os.path.join(ROOT, "paper_2604_05887_b200", "csrc", f), "rb").read())
+        text = open(os.path.join(ROOT, "paper_2604_05887_b200", "csrc", f)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(" ".join(text.split()).encode())
     return h.hexdigest()[:12]
 
 

@@ -24,7 +24,8 @@
 //     lower / upper bound of its scores); a CTA whose score barrier has received all bytes runs the
 //     same exact selection on its own copy (block_topk_blocked: one value histogram, exact ranking
 //     of the threshold bin, three block barriers), so that every CTA knows the ascending list of
-//     selected chunks without a round trip through global memory.  The lists later calls may ask
+//     selected chunks without a round trip through global memory.  Chunks above the threshold bin
+//     are requested from HBM into L2 as soon as that bin is known (short lists only).  The lists later calls may ask
 //     for (scores, ids, token count) are written to global memory only after the attention's first
 //     copies have been issued.
 //   every unit, attention:  the unit's token list (static: the compacted rows; dynamic: the rows of
@@ -32,8 +33,7 @@
 //     ranges.  Per tile:  S^T = K Q^T  (rows = tokens, columns = query heads, so the group shares
 //     every loaded KV tile and no tensor-core row is padding), online softmax in float32 (base-2
 //     exponent, accumulators rescaled only when a running maximum moves), P^T moved into operand
-//     layout with movmatrix,  O^T += V^T P^T.  A CTA with a short list asks L2 for its tiles beyond
-//     the first ring-full as soon as it knows them.
+//     layout with movmatrix,  O^T += V^T P^T.
 //   merge:  the warps of a CTA are combined in shared memory.  Groups up to 8: every CTA then sends
 //     each owner CTA its share of (m, l, O) into the owner's idle score area (st.async crediting the
 //     owner's merge barrier), and each owner, once its bytes are in, reduces its slice of the output
@@ -68,8 +68,9 @@ constexpr int kParkBytes = 16 * kParkStride * 4 + 128;               // one warp
 constexpr int kRecvMlOff = 6144;   // inside the score area: (m, l) of every sender and row, after the O slices
 static_assert(kMaxCluster * 8 * 8 + kRecvMlOff <= kSelSmemChunks * 4 && 8 * kHeadDim * 4 + 4 * 4 * kMaxCluster <= kRecvMlOff,
               "push-merge receive area fits the score area for groups up to 8");
-// A CTA with at most this many tiles asks L2 for the tiles beyond its first ring-full right away (short,
-// latency-bound lists); longer lists are bandwidth-bound and do better without the extra requests.
+// A dynamic unit whose CTAs get at most this many tiles each (a short, latency-bound list) asks L2 for the chunks
+// it is certain to select while the list is still being built; longer lists are bandwidth-bound and do better
+// without the extra requests.
 constexpr int kPrefetchMaxTiles = 2 * kDecStages + 2;
 
 constexpr int kMaxWarps = 8;                                         // consumer warps per CTA (8 for groups up to 8, 4 above)
