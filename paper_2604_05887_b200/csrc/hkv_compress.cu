@@ -232,7 +232,7 @@ constexpr uint32_t kKeepAlways = 0xFFFFFFFFu;   // no float's key (it would be a
 
 __global__ void __launch_bounds__(kKeepThreads)
     static_select_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text,
-                         int key_slots) {
+                         int key_slots, int skip_done) {
   __shared__ __align__(16) int scratch[kKeepScratchInts];
   __shared__ int s_ntext;
   extern __shared__ __align__(16) uint32_t skey[];   // key_slots entries: every token's role, computed once
@@ -249,6 +249,8 @@ __global__ void __launch_bounds__(kKeepThreads)
   int32_t* out = reinterpret_cast<int32_t*>(cache + u->idx_off);
   const int hist_end = C - w;   // tokens before the window
   const bool cached = C <= key_slots;
+  // after the cluster kernel: only the units it left (their count of kept tokens is still zero)
+  if (skip_done && reinterpret_cast<const int32_t*>(cache + hdr->n_valid_off)[uid] != 0) return;
 
   if (tid == 0) s_ntext = 0;
   __syncthreads();
@@ -329,6 +331,244 @@ __global__ void __launch_bounds__(kKeepThreads)
   if (tid == 0) {
     reinterpret_cast<int32_t*>(cache + hdr->n_valid_off)[uid] = emitted;
     if (emitted != budget) {
+      int32_t* err = reinterpret_cast<int32_t*>(cache + hdr->err_off);
+      atomicCAS(&err[0], 0, HKV_ERR_INDEX);
+      err[1] = kErrIndex;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same keep-set with one thread-block CLUSTER per static unit: the unit's tokens are cut into kSelCluster
+// contiguous slices, one per CTA, so that no SM walks a whole 32 K-token sequence alone.  Four cluster barriers:
+//   1. every CTA publishes its slice's statistics (text tokens before the window; smallest / largest score key
+//      among the text and among the visual tokens) -> all know which class is ranked, k, and the key range;
+//   2. local 1024-bin histograms of the ranked keys are complete -> every CTA adds up all eight (thread b reads
+//      bin b of every peer through distributed shared memory) and finds the threshold bin on its own copy;
+//   3. the threshold bin's items, (key, index), have been stored into every CTA's candidate list at slots that
+//      follow from the peers' counts of that bin -> every CTA ranks them exactly and knows the threshold element;
+//   4. the per-CTA numbers of selected tokens are known -> each CTA emits its ascending run at its offset.
+// Units this path does not take (a threshold bin with more than 1024 items, which needs the radix selection)
+// are left untouched: the single-CTA kernel, launched afterwards, does every unit whose count is still zero.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSelCluster = 8;
+struct __align__(16) SelStats { int n_text; uint32_t tmin, tmax, vmin, vmax; int pad[3]; };
+
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kKeepThreads)
+    static_select_cluster_kernel(char* cache, const char* workspace, const float* token_scores, const uint8_t* is_text,
+                                 int slice_slots) {
+  __shared__ __align__(16) int hist[kKeyedBins];
+  __shared__ __align__(16) uint2 cand[kKeepThreads];
+  __shared__ SelStats stats[kSelCluster];
+  __shared__ int counts[kSelCluster];
+  __shared__ int cnt_by_rank[kSelCluster];
+  __shared__ int ctl[8];
+  __shared__ int wtot[32];
+  extern __shared__ __align__(16) uint32_t skey[];          // slice_slots keys, then slice_slots text flags (bytes)
+  uint8_t* stxt = reinterpret_cast<uint8_t*>(skey + slice_slots);
+
+  const Header* hdr = reinterpret_cast<const Header*>(cache);
+  const uint32_t rank = cluster_ctarank();
+  int uid;
+  const Unit* u = unit_of(cache, hdr, false, blockIdx.x / kSelCluster, &uid);
+  const int C = u->C, w = hdr->obs_window, budget = u->n_tok;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint8_t* txt = is_text + static_cast<size_t>(u->b) * hdr->max_seq_len;
+  const float* scores = token_scores
+                            ? token_scores + (static_cast<size_t>(u->b) * hdr->n_kv_heads + u->h) * hdr->max_seq_len
+                            : reinterpret_cast<const float*>(workspace + u->ws_scores_off);
+  int32_t* out = reinterpret_cast<int32_t*>(cache + u->idx_off);
+  int32_t* n_valid = reinterpret_cast<int32_t*>(cache + hdr->n_valid_off) + uid;
+  const int hist_end = C - w;
+  const int per = (((C + kSelCluster - 1) / kSelCluster) + 3) & ~3;
+  const int lo = min(C, static_cast<int>(rank) * per), hi = min(C, lo + per), n = hi - lo;
+
+  if (budget <= w) {   // the last `budget` tokens, whatever their scores (uniform over the cluster)
+    const int start = C - budget;
+    for (int i = max(lo, start) + tid; i < hi; i += kKeepThreads) out[i - start] = i;
+    if (rank == 0 && tid == 0) *n_valid = budget;
+    return;
+  }
+
+  // ---- slice statistics ----
+  for (int i = tid; i < kKeyedBins; i += kKeepThreads) hist[i] = 0;
+  if (tid == 0) { ctl[0] = 0; ctl[1] = 0; ctl[4] = 0; ctl[5] = 0; }
+  int nt = 0;
+  uint32_t tmin = 0xFFFFFFFFu, tmax = 0u, vmin = 0xFFFFFFFFu, vmax = 0u;
+  for (int i = lo + tid; i < hi; i += kKeepThreads) {
+    const uint32_t kv = float_key(scores[i]);
+    const bool is_t = txt[i] != 0;
+    skey[i - lo] = kv;
+    stxt[i - lo] = is_t;
+    if (i < hist_end) {
+      if (is_t) { ++nt; tmin = min(tmin, kv); tmax = max(tmax, kv); }
+      else { vmin = min(vmin, kv); vmax = max(vmax, kv); }
+    }
+  }
+  nt = __reduce_add_sync(0xffffffffu, nt);
+  tmin = __reduce_min_sync(0xffffffffu, tmin); tmax = __reduce_max_sync(0xffffffffu, tmax);
+  vmin = __reduce_min_sync(0xffffffffu, vmin); vmax = __reduce_max_sync(0xffffffffu, vmax);
+  __shared__ SelStats mine;
+  if (tid == 0) mine = SelStats{0, 0xFFFFFFFFu, 0u, 0xFFFFFFFFu, 0u, {0, 0, 0}};
+  __syncthreads();
+  if (lane == 0) {
+    atomicAdd(&mine.n_text, nt);
+    atomicMin(&mine.tmin, tmin); atomicMax(&mine.tmax, tmax);
+    atomicMin(&mine.vmin, vmin); atomicMax(&mine.vmax, vmax);
+  }
+  __syncthreads();
+  if (tid < kSelCluster) {   // my statistics into slot `rank` of every CTA
+    const uint32_t dst = mapa(smem_u32(&stats[rank]), tid);
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(static_cast<uint32_t>(mine.n_text)),
+                 "r"(mine.tmin), "r"(mine.tmax), "r"(mine.vmin)
+                 : "memory");
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst + 16), "r"(mine.vmax) : "memory");
+  }
+  cluster_arrive(); cluster_wait();   // 1
+
+  int n_text = 0;
+  uint32_t kmin_t = 0xFFFFFFFFu, kmax_t = 0u, kmin_v = 0xFFFFFFFFu, kmax_v = 0u;
+#pragma unroll
+  for (int r = 0; r < kSelCluster; ++r) {
+    n_text += stats[r].n_text;
+    kmin_t = min(kmin_t, stats[r].tmin); kmax_t = max(kmax_t, stats[r].tmax);
+    kmin_v = min(kmin_v, stats[r].vmin); kmax_v = max(kmax_v, stats[r].vmax);
+  }
+  const int room = budget - w;
+  const bool rank_text = n_text >= room;       // window + text do not fit: rank the text tokens
+  const int k = rank_text ? room : room - n_text;
+  const uint32_t kmin = rank_text ? kmin_t : kmin_v, kmax = rank_text ? kmax_t : kmax_v;
+  const int shift = max(0, 32 - __clz((kmax - kmin) | 1u) - 10);
+  // roles of a token of my slice: ranked candidate / kept regardless / out
+  auto is_cand = [&](int j) { return lo + j < hist_end && (stxt[j] != 0) == rank_text; };
+  auto is_always = [&](int j) { return lo + j >= hist_end || (!rank_text && stxt[j] != 0); };
+
+  uint32_t tkey = 0xFFFFFFFFu;   // nothing ranked is taken unless the selection below says so
+  int tidx = -1;
+  if (k > 0) {
+    // ---- histograms ----
+    for (int j = tid; j < n; j += kKeepThreads)
+      if (is_cand(j)) atomicAdd(&hist[(skey[j] - kmin) >> shift], 1);
+    __syncthreads();
+    cluster_arrive(); cluster_wait();   // 2
+    int hr[kSelCluster], mine_tot = 0;
+    {
+      const uint32_t a = smem_u32(&hist[tid]);
+#pragma unroll
+      for (int r = 0; r < kSelCluster; ++r) {
+        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(hr[r]) : "r"(mapa(a, r)) : "memory");
+        mine_tot += hr[r];
+      }
+    }
+    // the highest bin b with count(bins > b) < k <= count(bins >= b): thread t owns bin t
+    {
+      int run = mine_tot;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_down_sync(0xffffffffu, run, off);
+        if (lane + off < 32) run += v;
+      }
+      if (lane == 0) wtot[warp] = run;
+      __syncthreads();
+      const int wt = wtot[lane];
+      int wrun = wt;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_down_sync(0xffffffffu, wrun, off);
+        if (lane + off < 32) wrun += v;
+      }
+      const int above = __shfl_sync(0xffffffffu, wrun - wt, warp) + run - mine_tot;
+      if (above < k && k <= above + mine_tot) {
+        ctl[1] = tid; ctl[2] = k - above; ctl[3] = mine_tot;
+#pragma unroll
+        for (int r = 0; r < kSelCluster; ++r) cnt_by_rank[r] = hr[r];
+      }
+      __syncthreads();
+    }
+    const int tbin = ctl[1], need = ctl[2], cnt = ctl[3];
+    if (cnt > kKeepThreads) {   // too many near-equal scores for the direct ranking: leave the unit to the general kernel
+      cluster_arrive(); cluster_wait();   // peers may still be reading my histogram
+      return;
+    }
+    // ---- the threshold bin's items into every CTA's candidate list ----
+    int base = 0;
+    for (int r = 0; r < static_cast<int>(rank); ++r) base += cnt_by_rank[r];
+    for (int j = tid; j < n; j += kKeepThreads) {
+      if (is_cand(j) && static_cast<int>((skey[j] - kmin) >> shift) == tbin) {
+        const int slot = base + atomicAdd(&ctl[0], 1);
+        const uint32_t a = smem_u32(&cand[slot]);
+#pragma unroll
+        for (int r = 0; r < kSelCluster; ++r)
+          asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(mapa(a, r)), "r"(skey[j]), "r"(static_cast<uint32_t>(lo + j))
+                       : "memory");
+      }
+    }
+    cluster_arrive(); cluster_wait();   // 3
+    if (tid < cnt) {
+      const uint2 me = cand[tid];
+      int rk = 0;
+      for (int j = 0; j < cnt; ++j) {
+        const uint2 o = cand[j];
+        rk += (o.x > me.x) || (o.x == me.x && o.y < me.y);
+      }
+      if (rk == need - 1) { ctl[4] = static_cast<int>(me.x); ctl[5] = static_cast<int>(me.y); }
+    }
+    __syncthreads();
+    tkey = static_cast<uint32_t>(ctl[4]);
+    tidx = ctl[5];
+  }
+
+  // ---- ordered emission: warp w owns a contiguous run of the slice ----
+  auto taken = [&](int j) {
+    if (is_always(j)) return true;
+    if (!is_cand(j)) return false;
+    const uint32_t kv = skey[j];
+    return kv > tkey || (kv == tkey && lo + j <= tidx);
+  };
+  constexpr int kWarps = kKeepThreads / 32;
+  const int wper = ((n + kWarps - 1) / kWarps + 31) & ~31;
+  const int beg = min(n, warp * wper), end = min(n, beg + wper);
+  int mine_n = 0;
+  for (int j0 = beg; j0 < end; j0 += 32) {
+    const int j = j0 + lane;
+    mine_n += __popc(__ballot_sync(0xffffffffu, j < end && taken(j)));
+  }
+  __syncthreads();   // wtot is free again
+  if (lane == 0) wtot[warp] = mine_n;
+  __syncthreads();
+  int before = 0, total = 0;
+  {
+    const int wt = wtot[lane];
+    int incl = wt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += v;
+    }
+    before = __shfl_sync(0xffffffffu, incl - wt, warp);
+    total = __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (tid < kSelCluster)
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa(smem_u32(&counts[rank]), tid)), "r"(total) : "memory");
+  cluster_arrive(); cluster_wait();   // 4
+  int off0 = 0, all = 0;
+#pragma unroll
+  for (int r = 0; r < kSelCluster; ++r) {
+    if (r < static_cast<int>(rank)) off0 += counts[r];
+    all += counts[r];
+  }
+  before += off0;
+  const uint32_t below = (1u << lane) - 1u;
+  for (int j0 = beg; j0 < end; j0 += 32) {
+    const int j = j0 + lane;
+    const bool sel = j < end && taken(j);
+    const uint32_t b = __ballot_sync(0xffffffffu, sel);
+    if (sel) out[before + __popc(b & below)] = lo + j;
+    before += __popc(b);
+  }
+  if (rank == 0 && tid == 0) {
+    *n_valid = all;
+    if (all != budget) {
       int32_t* err = reinterpret_cast<int32_t*>(cache + hdr->err_off);
       atomicCAS(&err[0], 0, HKV_ERR_INDEX);
       err[1] = kErrIndex;
@@ -504,6 +744,21 @@ cudaError_t launch_window_scores(char* cache, char* workspace, const void* k, co
 cudaError_t launch_static_select(char* cache, char* workspace, const float* token_scores, const uint8_t* is_text,
                                  const Header& hdr, cudaStream_t stream) {
   if (hdr.n_static == 0) return cudaSuccess;
+  // A cluster of kSelCluster CTAs per unit when a slice of the longest sequence (keys + text flags) fits one
+  // CTA's shared memory; the single-CTA kernel follows for the units the cluster kernel leaves (crowded threshold
+  // bin) and does everything for longer sequences.
+  const int slice = ((hdr.max_seq_len + kSelCluster - 1) / kSelCluster + 3) & ~3;
+  const size_t slice_smem = static_cast<size_t>(slice) * 5 + 16;
+  const bool clustered = slice_smem <= 160 * 1024;
+  if (clustered) {
+    cudaError_t e = cudaFuncSetAttribute(static_select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(slice_smem));
+    if (e != cudaSuccess) return e;
+    static_select_cluster_kernel<<<hdr.n_static * kSelCluster, kKeepThreads, slice_smem, stream>>>(
+        cache, workspace, token_scores, is_text, slice);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
   // every token's role is kept in shared memory when the longest sequence fits (else it is recomputed per pass)
   const int key_slots = std::min(hdr.max_seq_len, 49152);
   const size_t smem = static_cast<size_t>(key_slots) * sizeof(uint32_t);
@@ -511,7 +766,7 @@ cudaError_t launch_static_select(char* cache, char* workspace, const float* toke
       cudaFuncSetAttribute(static_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   static_select_kernel<<<hdr.n_static, kKeepThreads, smem, stream>>>(cache, workspace, token_scores, is_text,
-                                                                     key_slots);
+                                                                     key_slots, clustered ? 1 : 0);
   return cudaGetLastError();
 }
 
