@@ -30,6 +30,7 @@ constexpr int kClsRank = 256;          // largest threshold bin that is sorted d
 constexpr int kClsBins = 4096;          // bits 30..18 of a float in [0, 1]: 32 bins per octave
 constexpr int kClsShift = 18;
 constexpr int kClsLoadParts = 4;       // pieces a row arrives in, so that the maximum overlaps the copy
+constexpr int kClsRegVecs = 8;         // float4s of a row a thread keeps in registers (rows up to 32768 floats)
 constexpr int kClsRowScratch = (kClsBins + kClsRank + 32 + 8 + 32) * 4 + kClsLoadParts * 8;   // histogram, candidates, reduction slots, control words, warp sums, mbarriers
 
 struct ClsParams {
@@ -249,28 +250,79 @@ __global__ void __launch_bounds__(kClsRowThreads)
     for (int i = tid; i < kClsBins; i += kClsRowThreads) hist[i] = 0;
     if (tid == 0) ctl[3] = 0;
 
+    // Rows of up to kClsRegItems floats per thread stay in REGISTERS from the moment they land: the maximum, the
+    // probabilities, the histogram and the final sum are then computed without another trip through shared memory.
+    // Longer rows keep p in the row buffer (shared memory, or the workspace) and are walked again per pass.
+    const bool regs = staged && n4 <= kClsRegVecs * kClsRowThreads;
+    float4 rv[kClsRegVecs];
+    // visits every element this thread owns (p once the probabilities exist)
+    auto each = [&](auto fn) {
+      if (regs) {
+#pragma unroll
+        for (int q = 0; q < kClsRegVecs; ++q) {
+          if (q * kClsRowThreads + tid < n4) { fn(rv[q].x); fn(rv[q].y); fn(rv[q].z); fn(rv[q].w); }
+        }
+      } else {
+#pragma unroll 4
+        for (int i = tid; i < n4; i += kClsRowThreads) {
+          const float4 q = row4[i];
+          fn(q.x); fn(q.y); fn(q.z); fn(q.w);
+        }
+      }
+    };
+
     // maximum, piece by piece as the row lands; the up to three floats between C and the next
     // multiple of four become -inf, that is p = 0: zeros below every real entry, which no top-k
     // sum can feel
     float mx = -INFINITY;
     bool landed = true;
-    for (int part = 0; part < kClsLoadParts; ++part) {
-      const int beg = part * part4, end = min(n4, beg + part4);
-      if (beg >= end) break;
-      if (staged && landed) {
-        landed = mbar_wait_bounded(bar + part, (phases >> part) & 1u);
-        phases ^= 1u << part;
+    auto tail_fix = [&](float4& v, int i) {
+      if (i == n4 - 1 && (C & 3)) {
+        if ((C & 3) < 2) v.y = -INFINITY;
+        if ((C & 3) < 3) v.z = -INFINITY;
+        v.w = -INFINITY;
       }
-      if (!landed) continue;
-      for (int i = beg + tid; i < end; i += kClsRowThreads) {
-        float4 v = row4[i];
-        if (i == n4 - 1 && (C & 3)) {
-          if ((C & 3) < 2) v.y = -INFINITY;
-          if ((C & 3) < 3) v.z = -INFINITY;
-          v.w = -INFINITY;
-          row4[i] = v;
+    };
+    if (regs) {
+      uint32_t waited = 0u;
+#pragma unroll
+      for (int q = 0; q < kClsRegVecs; ++q) {
+        rv[q] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (q * kClsRowThreads < n4) {                       // the whole block of 1024 vectors lies in one piece
+          const int part = (q * kClsRowThreads) / part4;
+          if (landed && !((waited >> part) & 1u)) {
+            landed = mbar_wait_bounded(bar + part, (phases >> part) & 1u);
+            phases ^= 1u << part;
+            waited |= 1u << part;
+          }
+          const int i = q * kClsRowThreads + tid;
+          if (landed && i < n4) {
+            float4 v = row4[i];
+            tail_fix(v, i);
+            rv[q] = v;
+            mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+          }
         }
-        mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+      }
+      // pieces past the row's end were never armed; pieces armed but not visited cannot exist (every armed piece
+      // holds at least one block of vectors)
+    } else {
+      for (int part = 0; part < kClsLoadParts; ++part) {
+        const int beg = part * part4, end = min(n4, beg + part4);
+        if (beg >= end) break;
+        if (staged && landed) {
+          landed = mbar_wait_bounded(bar + part, (phases >> part) & 1u);
+          phases ^= 1u << part;
+        }
+        if (!landed) continue;
+        for (int i = beg + tid; i < end; i += kClsRowThreads) {
+          float4 v = row4[i];
+          if (i == n4 - 1 && (C & 3)) {
+            tail_fix(v, i);
+            row4[i] = v;
+          }
+          mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+        }
       }
     }
     if (__syncthreads_or(!landed)) {   // never seen; the whole CTA leaves, the row's sum and the score become NaN
@@ -286,16 +338,31 @@ __global__ void __launch_bounds__(kClsRowThreads)
       return fminf(q, 1.f);          // every bit pattern stays in [0, bits(1)]
     };
     float z = 0.f;
+    if (regs) {
+#pragma unroll
+      for (int q = 0; q < kClsRegVecs; ++q) {
+        if (q * kClsRowThreads + tid < n4) {
+          const float4 pq = make_float4(prob(rv[q].x), prob(rv[q].y), prob(rv[q].z), prob(rv[q].w));
+          rv[q] = pq;
+          z += (pq.x + pq.y) + (pq.z + pq.w);
+          atomicAdd(&hist[__float_as_uint(pq.x) >> kClsShift], 1);
+          atomicAdd(&hist[__float_as_uint(pq.y) >> kClsShift], 1);
+          atomicAdd(&hist[__float_as_uint(pq.z) >> kClsShift], 1);
+          atomicAdd(&hist[__float_as_uint(pq.w) >> kClsShift], 1);
+        }
+      }
+    } else {
 #pragma unroll 4
-    for (int i = tid; i < n4; i += kClsRowThreads) {
-      const float4 v = row4[i];
-      const float4 q = make_float4(prob(v.x), prob(v.y), prob(v.z), prob(v.w));
-      row4[i] = q;
-      z += (q.x + q.y) + (q.z + q.w);
-      atomicAdd(&hist[__float_as_uint(q.x) >> kClsShift], 1);
-      atomicAdd(&hist[__float_as_uint(q.y) >> kClsShift], 1);
-      atomicAdd(&hist[__float_as_uint(q.z) >> kClsShift], 1);
-      atomicAdd(&hist[__float_as_uint(q.w) >> kClsShift], 1);
+      for (int i = tid; i < n4; i += kClsRowThreads) {
+        const float4 v = row4[i];
+        const float4 q = make_float4(prob(v.x), prob(v.y), prob(v.z), prob(v.w));
+        row4[i] = q;
+        z += (q.x + q.y) + (q.z + q.w);
+        atomicAdd(&hist[__float_as_uint(q.x) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(q.y) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(q.z) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(q.w) >> kClsShift], 1);
+      }
     }
     const float Z = block_sum(z);   // its barriers also publish the histogram
     cls_find_bin(hist, kClsBins, k, ctl, wsum);
@@ -305,39 +372,25 @@ __global__ void __launch_bounds__(kClsRowThreads)
     float top = 0.f;
     for (;;) {
       if (need == cnt) {                      // the whole bin is inside the top k
-#pragma unroll 4
-        for (int i = tid; i < n4; i += kClsRowThreads) {
-          const float4 q = row4[i];
-          top += (((__float_as_uint(q.x) >> shift) >= prefix ? q.x : 0.f) +
-                  ((__float_as_uint(q.y) >> shift) >= prefix ? q.y : 0.f)) +
-                 (((__float_as_uint(q.z) >> shift) >= prefix ? q.z : 0.f) +
-                  ((__float_as_uint(q.w) >> shift) >= prefix ? q.w : 0.f));
-        }
+        each([&](float e) { top += (__float_as_uint(e) >> shift) >= prefix ? e : 0.f; });
+        break;
+      }
+      // A sharply peaked row: the k-th largest probability is so small that all `need` entries taken from its bin
+      // add up to less than 2^-26, while the sum holds the row's maximum p = 1 — they cannot move a float32 sum
+      // that is at least 1 by half a unit in the last place, so which of them count does not matter.
+      if (static_cast<float>(need) * __uint_as_float((prefix + 1u) << shift) < 1.4901161e-8f) {
+        each([&](float e) { top += (__float_as_uint(e) >> shift) > prefix ? e : 0.f; });
         break;
       }
       if (cnt <= kClsRank) {
-        // sum what lies above the bin, collect the bin's entries (a warp that meets some reserves
-        // their slots with one atomic) and sort them exactly (descending; equal values in an
+        // sum what lies above the bin, collect the bin's entries (each reserves its slot with one atomic; there
+        // are at most kClsRank of them in the whole row) and sort them exactly (descending; equal values in an
         // arbitrary but complete order): the first `need` join the sum
-#pragma unroll 4
-        for (int i0 = warp * 32; i0 < n4; i0 += kClsRowThreads) {
-          const int i = i0 + lane;
-          const float4 q = i < n4 ? row4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-          const float e[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint32_t hi = __float_as_uint(e[c]) >> shift;
-            if (hi > prefix) top += e[c];
-            const bool in_bin = i < n4 && hi == prefix;
-            const uint32_t m = __ballot_sync(0xffffffffu, in_bin);
-            if (m) {
-              int base = 0;
-              if (lane == 0) base = atomicAdd(&ctl[3], __popc(m));
-              base = __shfl_sync(0xffffffffu, base, 0);
-              if (in_bin) cand[base + __popc(m & ((1u << lane) - 1u))] = __float_as_uint(e[c]);
-            }
-          }
-        }
+        each([&](float e) {
+          const uint32_t hi = __float_as_uint(e) >> shift;
+          if (hi > prefix) top += e;
+          if (hi == prefix) cand[atomicAdd(&ctl[3], 1)] = __float_as_uint(e);
+        });
         __syncthreads();
         float* sorted = reinterpret_cast<float*>(hist);
         const int c = tid >> 2, part = tid & 3;          // four threads rank one entry
@@ -360,11 +413,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
         break;
       }
       if (shift == 0) {                       // more than kClsRank copies of one value: `need` of them count
-        for (int i = tid; i < n4; i += kClsRowThreads) {
-          const float4 q = row4[i];
-          top += ((__float_as_uint(q.x) > prefix ? q.x : 0.f) + (__float_as_uint(q.y) > prefix ? q.y : 0.f)) +
-                 ((__float_as_uint(q.z) > prefix ? q.z : 0.f) + (__float_as_uint(q.w) > prefix ? q.w : 0.f));
-        }
+        each([&](float e) { top += __float_as_uint(e) > prefix ? e : 0.f; });
         if (tid == 0) top += static_cast<float>(need) * __uint_as_float(prefix);
         break;
       }
@@ -374,14 +423,10 @@ __global__ void __launch_bounds__(kClsRowThreads)
       const uint32_t mask = (1u << width) - 1u;
       for (int i = tid; i < (1 << width); i += kClsRowThreads) hist[i] = 0;
       __syncthreads();
-      auto count = [&](float q) {
-        const uint32_t u = __float_as_uint(q);
+      each([&](float e) {
+        const uint32_t u = __float_as_uint(e);
         if ((u >> shift) == prefix) atomicAdd(&hist[(u >> nshift) & mask], 1);
-      };
-      for (int i = tid; i < n4; i += kClsRowThreads) {
-        const float4 q = row4[i];
-        count(q.x); count(q.y); count(q.z); count(q.w);
-      }
+      });
       __syncthreads();
       cls_find_bin(hist, 1 << width, need, ctl, wsum);
       __syncthreads();
