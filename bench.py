@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only without MEASURED_PEAKS.json
-NOMINAL_HBM_GBS = 8000.0           # the denominator the task statement names ("~8 TB/s")
+NOMINAL_HBM_GBS = 8000.0           # nominal HBM3e bandwidth of a B200, the second denominator reported
 N_LAYERS = {"cfg0": 1, "cfg1": 28, "cfg2": 28, "cfg3": 28, "cfg4": 1}
 N_QUERY_SETS = 8                   # distinct seeded queries per layer, rotated step by step
 STATS_REPLAYS = 500                # per-step CUDA-event pairs behind median / min / mean
