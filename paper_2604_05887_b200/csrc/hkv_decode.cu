@@ -81,8 +81,9 @@ constexpr int kScoresOff = kSelOff + kSelSmemChunks * 2;             // float32 
 constexpr int kBarsOff = kScoresOff + kSelSmemChunks * 4;            // mbarriers: ring stages, then scores, then merge
 constexpr int kScoreBar = kDecStages, kMergeBar = kDecStages + 1;
 constexpr int kArmedOff = kBarsOff + (kDecStages + 2) * 8;           // per stage: sequence number of the tile it was last armed with
-constexpr int kHistOff = kArmedOff + kDecStages * 4 + 8;             // selection: 256 bins
-constexpr int kBoundsOff = kHistOff + 256 * 4;                       // selection: (lower, upper) score bound of every warp of the cluster
+constexpr int kHistBins = 512;                                       // value bins of the selection (256 used for up to 512 chunks)
+constexpr int kHistOff = kArmedOff + kDecStages * 4 + 8;             // selection: histogram
+constexpr int kBoundsOff = kHistOff + kHistBins * 4;                       // selection: (lower, upper) score bound of every warp of the cluster
 constexpr int kCandOff = kBoundsOff;                                 // selection: 32 candidates (key, index); the bounds are dead by then
 constexpr int kMiscOff = kBoundsOff + kMaxCluster * kMaxWarps * 8;   // selection: counters
 constexpr int kSmemBytes = kMiscOff + 96;
@@ -222,7 +223,7 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
     }
     misc[0] = 0;
   }
-  if (exchange) { for (int i = tid; i < 256; i += W * 32) hist[i] = 0; }
+  if (exchange) { for (int i = tid; i < kHistBins; i += W * 32) hist[i] = 0; }
   // "this CTA is running and its barriers exist": has to be known before anybody touches its shared memory remotely
   if (clustered) cluster_arrive();
   bool bar_pending = clustered;   // an arrival on the cluster barrier that has not been waited for yet
@@ -569,10 +570,10 @@ __global__ void __launch_bounds__(W * 32, kDecCtasPerSm) decode_kernel(const __g
         const int ipt = (n_chunks + W * 32 - 1) / (W * 32);
         auto stamp = [&](int k2) { HKV_STAMP(20 + k2) };
         emitted = -1;
-        if (ipt <= 1) emitted = block_topk_blocked<W, 1>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
-        else if (ipt <= 2) emitted = block_topk_blocked<W, 2>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
-        else if (ipt <= 4) emitted = block_topk_blocked<W, 4>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
-        else if (ipt <= 8) emitted = block_topk_blocked<W, 8>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        if (ipt <= 1) emitted = block_topk_blocked<W, 1, 256>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 2) emitted = block_topk_blocked<W, 2, 256>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 4) emitted = block_topk_blocked<W, 4, 512>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
+        else if (ipt <= 8) emitted = block_topk_blocked<W, 8, 512>(sc_smem, n_chunks, n_mt * 16, k_sel, lo, hi, sel16, hist, cand, misc, early, stamp);
         if (emitted < 0) {
           // crowded threshold bin (or more scores than the fast path takes): the general selection, its
           // scratch in the idle ring

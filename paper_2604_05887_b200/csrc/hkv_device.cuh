@@ -436,7 +436,7 @@ __device__ int block_topk_smem(const float* scores, int n, int k, EmitFn emit, i
 // The decode step's fast path of the same selection: exact top-k over at most 256 * IPT finite float
 // scores in shared memory, three block barriers in all.  Thread t owns the IPT consecutive scores
 // [t * IPT, (t + 1) * IPT) in registers, so that the ascending output order is the thread order.
-//   1. every thread bins its scores into 256 equal-width value bins between lo and hi (lower and
+//   1. every thread bins its scores into NB (256 or 512) equal-width value bins between lo and hi (lower and
 //      upper bound of the scores, known to the caller) with shared-memory atomics        -> barrier
 //   2. every warp finds, redundantly, the bin of the k-th largest score; the scores of that bin are
 //      gathered as (key, index) candidates, and each warp publishes how many of its scores lie in
@@ -450,13 +450,14 @@ __device__ int block_topk_smem(const float* scores, int n, int k, EmitFn emit, i
 // Returns k, or -1 without having written anything when the threshold bin holds more than 32 scores
 // (many near-equal scores): the caller then runs block_topk_smem.  The decision is the same in
 // every thread.  Requires 1 <= k < n <= 256 * IPT, n_pad = n rounded up to a multiple of 16 readable
-// floats, blockDim.x = 32 * NWARPS with 256 * IPT >= n.  hist: 256 ints ZEROED by the caller, cand: 32 x (key, index), misc: 1 + NWARPS
+// floats, blockDim.x = 32 * NWARPS with 256 * IPT >= n.  hist: NB ints ZEROED by the caller, cand: 32 x (key, index), misc: 1 + NWARPS
 // ints with misc[0] ZEROED by the caller.
 // ---------------------------------------------------------------------------------------------
-template <int NWARPS, int IPT, class EarlyFn, class StampFn>
+template <int NWARPS, int IPT, int NB, class EarlyFn, class StampFn>
 __device__ int block_topk_blocked(const float* scores, int n, int n_pad, int k, float lo, float hi, uint16_t* out,
                                   int* hist, uint2* cand, int* misc, EarlyFn early, StampFn stamp) {
   static_assert(IPT == 1 || IPT == 2 || IPT == 4 || IPT == 8, "items per thread");
+  static_assert(NB == 256 || NB == 512, "value bins");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int i0 = tid * IPT;
   float v[IPT];
@@ -479,13 +480,13 @@ __device__ int block_topk_blocked(const float* scores, int n, int n_pad, int k, 
   }
   const float width = hi - lo;
   // the map score -> bin only has to be monotone, so an approximate quotient will do
-  const float scale = (width > 0.f && width < INFINITY) ? __fdividef(255.0f, width) : 0.f;
+  const float scale = (width > 0.f && width < INFINITY) ? __fdividef(static_cast<float>(NB - 1), width) : 0.f;
   int bin[IPT];
 #pragma unroll
   for (int e = 0; e < IPT; ++e) {
     bin[e] = -1;   // not an item
     if (i0 + e < n) {
-      bin[e] = max(0, min(255, __float2int_rd((v[e] - lo) * scale)));
+      bin[e] = max(0, min(NB - 1, __float2int_rd((v[e] - lo) * scale)));
       atomicAdd(&hist[bin[e]], 1);
     }
   }
@@ -495,11 +496,16 @@ __device__ int block_topk_blocked(const float* scores, int n, int n_pad, int k, 
   // every warp: the highest bin b with count(bins > b) < k <= count(bins >= b)
   int tbin, need, cnt;
   {
-    const int4 h0 = reinterpret_cast<const int4*>(hist)[lane * 2], h1 = reinterpret_cast<const int4*>(hist)[lane * 2 + 1];
-    const int loc[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+    constexpr int PER = NB / 32;   // bins per lane
+    int loc[PER];
+#pragma unroll
+    for (int q = 0; q < PER / 4; ++q) {
+      const int4 h = reinterpret_cast<const int4*>(hist)[lane * (PER / 4) + q];
+      loc[4 * q] = h.x; loc[4 * q + 1] = h.y; loc[4 * q + 2] = h.z; loc[4 * q + 3] = h.w;
+    }
     int tot = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) tot += loc[j];
+    for (int j = 0; j < PER; ++j) tot += loc[j];
     int run = tot;   // becomes the sum over lanes >= this one
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -512,8 +518,8 @@ __device__ int block_topk_blocked(const float* scores, int n, int n_pad, int k, 
     if (mine) {
       int acc = above;
 #pragma unroll
-      for (int j = 7; j >= 0; --j) {
-        if (acc < k && k <= acc + loc[j]) { my_bin = lane * 8 + j; my_need = k - acc; my_cnt = loc[j]; }
+      for (int j = PER - 1; j >= 0; --j) {
+        if (acc < k && k <= acc + loc[j]) { my_bin = lane * PER + j; my_need = k - acc; my_cnt = loc[j]; }
         acc += loc[j];
       }
     }
