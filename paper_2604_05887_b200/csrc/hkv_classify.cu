@@ -8,7 +8,9 @@
 //                      float32 into the workspace (rows padded to a multiple of 128 floats);
 //   cls_row_kernel     one CTA per row: the row in shared memory, max, p = 2^(l - max), normaliser,
 //                      the exact k-th largest p (histogram over the float bits, then exact ranking
-//                      of the threshold bin), the sum of the entries above it plus the tied share;
+//                      of the threshold bin), the sum of the entries above it plus the tied share
+//                      (cls_row_regs_kernel when no row of the group is longer than 32768 entries:
+//                      the row in registers, the next row's copy in flight meanwhile);
 //   cls_finish_kernel  (after the last pass) mean of the rows' sums in double, fixed order, and
 //                      the label.
 #include <algorithm>
@@ -255,20 +257,32 @@ __global__ void __launch_bounds__(kClsRowThreads)
     // Longer rows keep p in the row buffer (shared memory, or the workspace) and are walked again per pass.
     const bool regs = staged && n4 <= kClsRegVecs * kClsRowThreads;
     float4 rv[kClsRegVecs];
-    // visits every element this thread owns (p once the probabilities exist)
-    auto each = [&](auto fn) {
+    // visits every float4 this thread owns (p once the probabilities exist)
+    auto each4 = [&](auto fn) {
       if (regs) {
 #pragma unroll
         for (int q = 0; q < kClsRegVecs; ++q) {
-          if (q * kClsRowThreads + tid < n4) { fn(rv[q].x); fn(rv[q].y); fn(rv[q].z); fn(rv[q].w); }
+          if (q * kClsRowThreads + tid < n4) fn(rv[q]);
         }
       } else {
 #pragma unroll 4
-        for (int i = tid; i < n4; i += kClsRowThreads) {
-          const float4 q = row4[i];
-          fn(q.x); fn(q.y); fn(q.z); fn(q.w);
-        }
+        for (int i = tid; i < n4; i += kClsRowThreads) fn(row4[i]);
       }
+    };
+    auto each = [&](auto fn) {
+      each4([&](const float4& v) { fn(v.x); fn(v.y); fn(v.z); fn(v.w); });
+    };
+    // top += every entry whose bit pattern is at least `from` (the bits of a float in [0, 1] order like its value);
+    // four independent partial sums, added in a fixed order
+    auto add_from = [&](uint32_t from) {
+      float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+      each4([&](const float4& v) {
+        t0 += __float_as_uint(v.x) >= from ? v.x : 0.f;
+        t1 += __float_as_uint(v.y) >= from ? v.y : 0.f;
+        t2 += __float_as_uint(v.z) >= from ? v.z : 0.f;
+        t3 += __float_as_uint(v.w) >= from ? v.w : 0.f;
+      });
+      return (t0 + t1) + (t2 + t3);
     };
 
     // maximum, piece by piece as the row lands; the up to three floats between C and the next
@@ -284,12 +298,14 @@ __global__ void __launch_bounds__(kClsRowThreads)
       }
     };
     if (regs) {
+      static_assert(kClsLoadParts == 4, "piece index by three comparisons");
+      const int m4 = part4 / kClsRowThreads;   // blocks of kClsRowThreads vectors per piece
       uint32_t waited = 0u;
 #pragma unroll
       for (int q = 0; q < kClsRegVecs; ++q) {
         rv[q] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         if (q * kClsRowThreads < n4) {                       // the whole block of 1024 vectors lies in one piece
-          const int part = (q * kClsRowThreads) / part4;
+          const int part = (q >= m4) + (q >= 2 * m4) + (q >= 3 * m4);   // = q * kClsRowThreads / part4
           if (landed && !((waited >> part) & 1u)) {
             landed = mbar_wait_bounded(bar + part, (phases >> part) & 1u);
             phases ^= 1u << part;
@@ -333,9 +349,8 @@ __global__ void __launch_bounds__(kClsRowThreads)
 
     // p, normaliser, histogram
     auto prob = [&](float l) {
-      float q = fast_exp2(l - M);
-      if (!(q >= 0.f)) q = 0.f;      // a NaN logit counts as no attention
-      return fminf(q, 1.f);          // every bit pattern stays in [0, bits(1)]
+      // a NaN logit counts as no attention (fmaxf returns its other operand); every bit pattern stays in [0, bits(1)]
+      return fminf(fmaxf(fast_exp2(l - M), 0.f), 1.f);
     };
     float z = 0.f;
     if (regs) {
@@ -371,25 +386,32 @@ __global__ void __launch_bounds__(kClsRowThreads)
     int shift = kClsShift, need = ctl[1], cnt = ctl[2];
     float top = 0.f;
     for (;;) {
+      const uint32_t bin_lo = prefix << shift, bin_span = 1u << shift;   // the bin = bit patterns [bin_lo, bin_lo + bin_span)
       if (need == cnt) {                      // the whole bin is inside the top k
-        each([&](float e) { top += (__float_as_uint(e) >> shift) >= prefix ? e : 0.f; });
+        top = add_from(bin_lo);
         break;
       }
       // A sharply peaked row: the k-th largest probability is so small that all `need` entries taken from its bin
       // add up to less than 2^-26, while the sum holds the row's maximum p = 1 — they cannot move a float32 sum
       // that is at least 1 by half a unit in the last place, so which of them count does not matter.
       if (static_cast<float>(need) * __uint_as_float((prefix + 1u) << shift) < 1.4901161e-8f) {
-        each([&](float e) { top += (__float_as_uint(e) >> shift) > prefix ? e : 0.f; });
+        top = add_from(bin_lo + bin_span);
         break;
       }
       if (cnt <= kClsRank) {
         // sum what lies above the bin, collect the bin's entries (each reserves its slot with one atomic; there
         // are at most kClsRank of them in the whole row) and sort them exactly (descending; equal values in an
         // arbitrary but complete order): the first `need` join the sum
-        each([&](float e) {
-          const uint32_t hi = __float_as_uint(e) >> shift;
-          if (hi > prefix) top += e;
-          if (hi == prefix) cand[atomicAdd(&ctl[3], 1)] = __float_as_uint(e);
+        top = add_from(bin_lo + bin_span);
+        each4([&](const float4& v) {
+          const uint32_t a = __float_as_uint(v.x) - bin_lo, b = __float_as_uint(v.y) - bin_lo,
+                         c = __float_as_uint(v.z) - bin_lo, d = __float_as_uint(v.w) - bin_lo;
+          if (min(min(a, b), min(c, d)) < bin_span) {   // rare: at most kClsRank entries of the row pass
+            if (a < bin_span) cand[atomicAdd(&ctl[3], 1)] = a + bin_lo;
+            if (b < bin_span) cand[atomicAdd(&ctl[3], 1)] = b + bin_lo;
+            if (c < bin_span) cand[atomicAdd(&ctl[3], 1)] = c + bin_lo;
+            if (d < bin_span) cand[atomicAdd(&ctl[3], 1)] = d + bin_lo;
+          }
         });
         __syncthreads();
         float* sorted = reinterpret_cast<float*>(hist);
@@ -413,7 +435,7 @@ __global__ void __launch_bounds__(kClsRowThreads)
         break;
       }
       if (shift == 0) {                       // more than kClsRank copies of one value: `need` of them count
-        each([&](float e) { top += __float_as_uint(e) > prefix ? e : 0.f; });
+        top = add_from(prefix + 1u);
         if (tid == 0) top += static_cast<float>(need) * __uint_as_float(prefix);
         break;
       }
@@ -437,6 +459,316 @@ __global__ void __launch_bounds__(kClsRowThreads)
     }
     top = block_sum(top);
     if (tid == 0) rowsum[static_cast<size_t>(unit) * P.r_stride + r] = top / Z;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same row sums for rows of up to kClsRegCols entries, every entry in a register of the CTA
+// (kClsRegThreads threads x 32 entries), as a two-row pipeline: a row lands in shared memory in
+// pieces of one vector per thread, each on its own mbarrier; once every thread has taken its
+// entries into registers (the first block barrier of the row) one thread starts the NEXT row's
+// copies into the same buffer, so they travel while this row's probabilities, histogram,
+// threshold and sums are computed.  That thread also works out where the next row lies and hands
+// it over through a two-slot descriptor in shared memory.  Arithmetic as in cls_row_kernel; sums in
+// a fixed order.  (Measured and dropped: 512 threads of 64 entries -- a sixth fewer instructions,
+// but a quarter slower with half the warps to hide latency; the threshold bin ranked by one warp
+// after the last barrier -- slower than ranking it with the whole block between two barriers.)
+// ---------------------------------------------------------------------------------------------
+constexpr int kClsRegCols = 32768;
+constexpr int kClsRegThreads = 1024;   // 512 threads x 128 entries issue a sixth fewer instructions but hide less latency: slower
+constexpr int kClsRegWarps = kClsRegThreads / 32;
+constexpr int kClsRegVecsT = kClsRegCols / 4 / kClsRegThreads;   // float4s per thread: 16
+// histogram, candidates, their sorted copy, three reduction slots, control words, warp sums, two row descriptors,
+// piece barriers
+constexpr int kClsRegScratch = (kClsBins + 2 * kClsRank + 3 * 32 + 8 + 32 + 2 * 8) * 4 + kClsRegVecsT * 8;
+static_assert(kClsRegScratch % 16 == 0, "the row buffer is 16-byte aligned");
+constexpr int kClsRegBinsPer = kClsBins / kClsRegThreads;   // bins a thread sums in the threshold search
+static_assert((kClsRegBinsPer == 4 || kClsRegBinsPer == 8) && kClsRegVecsT <= 32, "whole int4s of bins per thread; one phase bit per piece");
+
+// cls_find_bin for a block of kClsRegThreads threads (nbins 4096, 1024 or 256).
+__device__ __forceinline__ void cls_find_bin_regs(const int* hist, int nbins, int need, int* ctl, int* wsum) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = nbins == kClsBins ? kClsRegBinsPer : nbins > kClsRegThreads ? nbins / kClsRegThreads : 1;   // 4 or 8; 2 or 1; 1
+  int loc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (nbins == kClsBins) {
+    const int4 u = reinterpret_cast<const int4*>(hist)[tid * (kClsRegBinsPer / 4)];
+    loc[0] = u.x; loc[1] = u.y; loc[2] = u.z; loc[3] = u.w;
+    if (kClsRegBinsPer == 8) {
+      const int4 v = reinterpret_cast<const int4*>(hist)[tid * 2 + 1];
+      loc[4] = v.x; loc[5] = v.y; loc[6] = v.z; loc[7] = v.w;
+    }
+  } else if (per == 2) {
+    const int2 u = reinterpret_cast<const int2*>(hist)[tid];
+    loc[0] = u.x; loc[1] = u.y;
+  } else if (tid < nbins) {
+    loc[0] = hist[tid];
+  }
+  const int tot = ((loc[0] + loc[1]) + (loc[2] + loc[3])) + ((loc[4] + loc[5]) + (loc[6] + loc[7]));
+  int run = tot;   // becomes the sum over this and the higher lanes of the warp
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_down_sync(0xffffffffu, run, off);
+    if (lane + off < 32) run += v;
+  }
+  if (lane == 0) wsum[warp] = run;
+  __syncthreads();
+  const int wt = lane < kClsRegWarps ? wsum[lane] : 0;
+  int wrun = wt;   // sum over warps >= lane
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_down_sync(0xffffffffu, wrun, off);
+    if (lane + off < 32) wrun += v;
+  }
+  int acc = __shfl_sync(0xffffffffu, wrun - wt, warp) + run - tot;   // items in the bins above this thread's
+  if (acc < need && need <= acc + tot) {
+#pragma unroll
+    for (int j = 7; j >= 0; --j) {
+      if (j < per && acc < need && need <= acc + loc[j]) {
+        ctl[0] = tid * per + j;
+        ctl[1] = need - acc;
+        ctl[2] = loc[j];
+      }
+      if (j < per) acc += loc[j];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kClsRegThreads)
+    cls_row_regs_kernel(const ClsParams P, const float* logits, float* rowsum, int rows_pass, int total_rows) {
+  extern __shared__ __align__(16) uint8_t cls_smem[];
+  int* hist = reinterpret_cast<int*>(cls_smem);                   // [kClsBins]
+  uint32_t* cand = reinterpret_cast<uint32_t*>(hist + kClsBins);  // [kClsRank]
+  float* sorted = reinterpret_cast<float*>(cand + kClsRank);      // [kClsRank]: the threshold bin in descending order
+  float* red = sorted + kClsRank;                                 // [3][32]: one slot per reduction of a row
+  int* ctl = reinterpret_cast<int*>(red + 3 * 32);                // [8]
+  int* wsum = ctl + 8;                                            // [32]
+  int* desc = wsum + 32;                                          // [2][8]: idx (-1: none), unit, C, r, k, offset lo, hi
+  uint64_t* bar = reinterpret_cast<uint64_t*>(desc + 16);         // [kClsRegVecsT]
+  float4* srow4 = reinterpret_cast<float4*>(cls_smem + kClsRegScratch);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // thread 0 only: the first row at or after `idx` (stride gridDim.x) that exists -> descriptor slot, and its copies
+  auto post_row = [&](int idx, int slot) {
+    int* d = desc + slot * 8;
+    for (; idx < total_rows; idx += gridDim.x) {
+      const int unit = idx / rows_pass, rr = idx - unit * rows_pass, b = unit / P.n_kv_heads;
+      const int r = P.row_begin + rr;
+      if (r >= P.T[b] * P.group) continue;      // a short sequence does not have this row
+      const int C = P.C[b];
+      const size_t off = (static_cast<size_t>(unit) * P.row_block + rr) * P.c_stride;
+      d[0] = idx; d[1] = unit; d[2] = C; d[3] = r; d[4] = P.k[b];
+      const int n4 = (C + 3) >> 2;
+      // whole 16-byte pieces: rows start 256-byte aligned and are padded to a multiple of 128 floats
+      fence_proxy_async();
+      const float4* src = reinterpret_cast<const float4*>(logits + off);
+      for (int q = 0; q * kClsRegThreads < n4; ++q) {
+        const uint32_t bytes = static_cast<uint32_t>(min(kClsRegThreads, n4 - q * kClsRegThreads)) * 16u;
+        mbar_arrive_expect_tx(bar + q, bytes);
+        bulk_g2s(srow4 + q * kClsRegThreads, src + q * kClsRegThreads, bytes, bar + q);
+      }
+      return;
+    }
+    d[0] = -1;
+  };
+
+  if (tid == 0) {
+    for (int i = 0; i < kClsRegVecsT; ++i) mbar_init(bar + i, 1);
+    mbar_fence_init();
+    ctl[3] = 0;
+    post_row(blockIdx.x, 0);
+  }
+  for (int i = tid; i < kClsBins; i += kClsRegThreads) hist[i] = 0;
+  __syncthreads();
+  uint32_t phases = 0;   // bit q: parity the next wait on barrier q looks for
+
+  for (int it = 0;; ++it) {
+    const int* d = desc + (it & 1) * 8;
+    const int idx = d[0];
+    if (idx < 0) break;
+    const int unit = d[1], C = d[2], r = d[3], k = d[4];
+    const int n4 = (C + 3) >> 2;
+
+    // the row's entries into registers, piece by piece as they land, with the running maximum; the up to three
+    // floats between C and the next multiple of four become -inf, that is p = 0: zeros below every real entry,
+    // which no top-k sum can feel
+    float4 rv[kClsRegVecsT];   // rv[q] is used only where q * kClsRegThreads + tid < n4
+    float mx = -INFINITY;
+    bool landed = true;
+    const int i_fix = (C & 3) ? n4 - 1 : -1;   // the vector with floats past the row's end
+#pragma unroll
+    for (int q = 0; q < kClsRegVecsT; ++q) {
+      if (q * kClsRegThreads < n4) {
+        if (landed) landed = mbar_wait_bounded(bar + q, (phases >> q) & 1u);
+        phases ^= 1u << q;
+        const int i = q * kClsRegThreads + tid;
+        if (landed && i < n4) {
+          float4 v = srow4[i];
+          if (i == i_fix) {
+            if ((C & 3) < 2) v.y = -INFINITY;
+            if ((C & 3) < 3) v.z = -INFINITY;
+            v.w = -INFINITY;
+          }
+          rv[q] = v;
+          mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+        }
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if (lane == 0) red[warp] = mx;
+    // every thread holds its entries: the buffer is free.  A wait that ran out (never seen): the whole CTA
+    // leaves, the row's sum and with it the unit's score become NaN
+    if (__syncthreads_or(!landed)) {
+      if (tid == 0) rowsum[static_cast<size_t>(unit) * P.r_stride + r] = __int_as_float(0x7FC00000);
+      return;
+    }
+    if (tid == 0) post_row(idx + gridDim.x, (it + 1) & 1);   // the next row travels during the rest of this one
+    float M = lane < kClsRegWarps ? red[lane] : -INFINITY;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+
+    // p = 2^(l - max) in [0, 1] (a NaN logit counts as no attention: fmaxf returns its other operand), the
+    // normaliser, and the histogram over bits 30..18 of p
+    float z = 0.f;
+#pragma unroll
+    for (int q = 0; q < kClsRegVecsT; ++q) {
+      if (q * kClsRegThreads + tid < n4) {
+        float4 pq;
+        pq.x = fminf(fmaxf(fast_exp2(rv[q].x - M), 0.f), 1.f);
+        pq.y = fminf(fmaxf(fast_exp2(rv[q].y - M), 0.f), 1.f);
+        pq.z = fminf(fmaxf(fast_exp2(rv[q].z - M), 0.f), 1.f);
+        pq.w = fminf(fmaxf(fast_exp2(rv[q].w - M), 0.f), 1.f);
+        rv[q] = pq;
+        z += (pq.x + pq.y) + (pq.z + pq.w);
+        atomicAdd(&hist[__float_as_uint(pq.x) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(pq.y) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(pq.z) >> kClsShift], 1);
+        atomicAdd(&hist[__float_as_uint(pq.w) >> kClsShift], 1);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+    if (lane == 0) red[32 + warp] = z;
+    __syncthreads();   // publishes the warp sums and the histogram
+    float Z = lane < kClsRegWarps ? red[32 + lane] : 0.f;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
+    cls_find_bin_regs(hist, kClsBins, k, ctl, wsum);
+    __syncthreads();
+    auto each4 = [&](auto fn) {
+#pragma unroll
+      for (int q = 0; q < kClsRegVecsT; ++q) {
+        if (q * kClsRegThreads + tid < n4) fn(rv[q]);
+      }
+    };
+    // the sum of every entry whose bit pattern is at least `from`; four partial sums added in a fixed order
+    auto add_from = [&](uint32_t from) {
+      float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+      each4([&](const float4& v) {
+        t0 += __float_as_uint(v.x) >= from ? v.x : 0.f;
+        t1 += __float_as_uint(v.y) >= from ? v.y : 0.f;
+        t2 += __float_as_uint(v.z) >= from ? v.z : 0.f;
+        t3 += __float_as_uint(v.w) >= from ? v.w : 0.f;
+      });
+      return (t0 + t1) + (t2 + t3);
+    };
+    // the entries with bit patterns in [lo, lo + span) each reserve a slot of cand[] (the caller knows their number)
+    auto collect = [&](uint32_t lo, uint32_t span) {
+      each4([&](const float4& v) {
+        const uint32_t a = __float_as_uint(v.x) - lo, b = __float_as_uint(v.y) - lo, c = __float_as_uint(v.z) - lo,
+                       e = __float_as_uint(v.w) - lo;
+        if (min(min(a, b), min(c, e)) < span) {
+          if (a < span) cand[atomicAdd(&ctl[3], 1)] = a + lo;
+          if (b < span) cand[atomicAdd(&ctl[3], 1)] = b + lo;
+          if (c < span) cand[atomicAdd(&ctl[3], 1)] = c + lo;
+          if (e < span) cand[atomicAdd(&ctl[3], 1)] = e + lo;
+        }
+      });
+    };
+    uint32_t prefix = static_cast<uint32_t>(ctl[0]);
+    int shift = kClsShift, need = ctl[1], cnt = ctl[2];
+    float top = 0.f;
+    int n_sorted = 0;   // entries of sorted[] that belong to the sum
+    for (;;) {
+      const uint32_t bin_lo = prefix << shift, bin_span = 1u << shift;   // the bin = bit patterns [bin_lo, bin_lo + bin_span)
+      if (need == cnt) {                      // the whole bin is inside the top k
+        top = add_from(bin_lo);
+        break;
+      }
+      // A sharply peaked row: all `need` entries taken from the bin add up to less than 2^-26 while the sum holds
+      // the row's maximum p = 1, so they cannot move it by half a unit in the last place
+      if (static_cast<float>(need) * __uint_as_float(bin_lo + bin_span) < 1.4901161e-8f) {
+        top = add_from(bin_lo + bin_span);
+        break;
+      }
+      if (cnt <= kClsRank) {
+        // up to kClsRank entries: ranked exactly (descending; equal values in an arbitrary but complete order) by
+        // several threads per entry; warp 0 adds the first `need` in that order after the row's last barrier
+        top = add_from(bin_lo + bin_span);
+        collect(bin_lo, bin_span);
+        __syncthreads();
+        constexpr int kSh = kClsRegThreads == 1024 ? 2 : 1;   // log2 of threads per entry when all kClsRank slots are in use
+        const int sh = cnt <= kClsRank / 2 ? kSh + 1 : kSh;
+        const int c = tid >> sh, part = tid & ((1 << sh) - 1);
+        const uint32_t mk = c < cnt ? cand[c] : 0u;
+        int rank = 0;   // entries that come before this one
+        if (c < cnt) {
+          for (int j = part; j < cnt; j += 1 << sh) {
+            const uint32_t o = cand[j];
+            rank += (o > mk) || (o == mk && j < c);
+          }
+        }
+        for (int off = 1; off < (1 << sh); off <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, off);
+        if (c < cnt && part == 0) sorted[rank] = __uint_as_float(mk);
+        n_sorted = need;
+        break;
+      }
+      if (shift == 0) {                       // more than kClsRank copies of one value: `need` of them count
+        top = add_from(prefix + 1u);
+        if (tid == 0) top += static_cast<float>(need) * __uint_as_float(prefix);
+        break;
+      }
+      // a crowded bin: histogram of the next bits of its entries (17..8, then 7..0)
+      const int width = shift == kClsShift ? 10 : 8;
+      const int nshift = shift - width;
+      const uint32_t mask = (1u << width) - 1u;
+      for (int i = tid; i < (1 << width); i += kClsRegThreads) hist[i] = 0;
+      __syncthreads();
+      each4([&](const float4& v) {
+        const uint32_t u[4] = {__float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if ((u[e] >> shift) == prefix) atomicAdd(&hist[(u[e] >> nshift) & mask], 1);
+      });
+      __syncthreads();
+      cls_find_bin_regs(hist, 1 << width, need, ctl, wsum);
+      __syncthreads();
+      prefix = (prefix << width) | static_cast<uint32_t>(ctl[0]);
+      shift = nshift;
+      need = ctl[1];
+      cnt = ctl[2];
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) top += __shfl_xor_sync(0xffffffffu, top, off);
+    if (lane == 0) red[64 + warp] = top;
+    __syncthreads();   // every reader of the histogram area and of the control words is done
+    if (warp == 0) {
+      float t = lane < kClsRegWarps ? red[64 + lane] : 0.f;
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+      if (n_sorted > 0) {   // the threshold bin's share, largest first, in a fixed order
+        float s = 0.f;
+        for (int j = lane; j < n_sorted; j += 32) s += sorted[j];
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        t += s;
+      }
+      if (lane == 0) {
+        rowsum[static_cast<size_t>(unit) * P.r_stride + r] = t / Z;
+        ctl[3] = 0;
+      }
+    }
+    for (int i = tid; i < kClsBins; i += kClsRegThreads) hist[i] = 0;   // for the next row; its first barrier orders it
   }
 }
 
@@ -545,6 +877,10 @@ extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, c
   if (cudaFuncSetAttribute(cls_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            static_cast<int>(row_smem)) != cudaSuccess)
     return HKV_ERR_CUDA;
+  const size_t regs_smem = kClsRegScratch + static_cast<size_t>(kClsRegCols) * sizeof(float);
+  if (cudaFuncSetAttribute(cls_row_regs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(regs_smem)) != cudaSuccess)
+    return HKV_ERR_CUDA;
 
   int dev = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -599,7 +935,11 @@ extern "C" hkv_status hkv_classify_heads(const hkv_config* cfg, const void* k, c
       cls_logits_tc_kernel<<<dim3((n_tiles + tiles_per_cta - 1) / tiles_per_cta, row_blocks, units), tc::kThreads,
                              tc::kSmemBytes, cs>>>(P, kg, qg, logits, tiles_per_cta, err);
       const int total_rows = rows * units;
-      cls_row_kernel<<<std::min(total_rows, n_sm), kClsRowThreads, row_smem, cs>>>(P, logits, rowsum, rows, total_rows);
+      if (cg_max <= kClsRegCols)   // every row of the group fits the threads' registers: the pipelined kernel
+        cls_row_regs_kernel<<<std::min(total_rows, n_sm), kClsRegThreads, regs_smem, cs>>>(P, logits, rowsum, rows,
+                                                                                           total_rows);
+      else
+        cls_row_kernel<<<std::min(total_rows, n_sm), kClsRowThreads, row_smem, cs>>>(P, logits, rowsum, rows, total_rows);
     }
     cls_finish_kernel<<<units, 256, 0, cs>>>(P, rowsum, err, theta, scores_out, head_type_out, b0 * cfg->n_kv_heads);
     if (cudaGetLastError() != cudaSuccess) return HKV_ERR_CUDA;
