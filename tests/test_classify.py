@@ -139,6 +139,25 @@ def test_gpu_classify_several_row_blocks_in_one_pass():
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("C", [32768, 32765, 31745, 1023, 5])
+def test_gpu_classify_rows_kept_in_registers(C):
+    """Rows of up to 32768 entries take the pipelined kernel (the row in registers, the next row's copy in flight):
+    the longest such row, lengths that are no multiple of four, a last piece of one vector, rows shorter than one
+    piece, and rows of a handful of entries."""
+    L = hi.tiny(seed=41, B=2 if C < 2000 else 1, C=C, chunk_size=32 if C >= 64 else 1, w=8 if C >= 64 else 2, Hq=8, Hkv=2,
+                d=128, ragged=False)
+    _check_case(L, 5, 0.05)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("C", [32769, 49152])
+def test_gpu_classify_rows_kept_in_shared_memory(C):
+    """Between 32769 and 49152 entries a row stays in shared memory (the general kernel), beyond that in the workspace."""
+    L = hi.tiny(seed=42, B=1, C=C, chunk_size=32, w=8, Hq=4, Hkv=2, d=128, ragged=False)
+    _check_case(L, 3, 0.05)
+
+
+@pytest.mark.gpu
 def test_gpu_classify_rows_longer_than_shared_memory():
     L = hi.tiny(seed=33, B=1, C=50021, chunk_size=32, w=8, Hq=8, Hkv=2, d=128)
     _check_case(L, 3, 0.05)
