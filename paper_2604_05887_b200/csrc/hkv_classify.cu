@@ -48,9 +48,10 @@ struct ClsParams {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Logits (tcgen05 tensor cores, accumulators in tensor memory).  One CTA = 256 rows of one unit (two accumulator blocks) x a range of
-// 128-key tiles; a draining warp owns 32 rows of one block and 64 of the tile's keys and writes them
-// in 64-byte runs.  grid (key ranges, 256-row blocks of the pass, units).
+// Logits (tcgen05 tensor cores, accumulators in tensor memory).  One CTA = 256 rows of one unit x a range of
+// 128-key tiles; the tile's keys are the accumulator's rows (lanes) and the 256 query rows its columns, so a
+// draining warp owns 32 consecutive keys and 64 rows and writes, per row, one 128-byte line.
+// grid (key ranges, 256-row blocks of the pass, units).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(tc::kThreads, 1)
     cls_logits_tc_kernel(const ClsParams P, const __nv_bfloat16* kin, const __nv_bfloat16* q_text, float* logits,
@@ -74,38 +75,31 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
       kin + (static_cast<size_t>(b) * P.n_kv_heads + h) * static_cast<size_t>(P.max_seq_len) * kHeadDim;
   float* out = logits + static_cast<size_t>(unit) * P.row_block * P.c_stride;
   const float sc = P.scale_log2e;
-  auto epilogue = [&](int tile, int lane_row, int part, auto groups, float* scratch, auto, uint64_t*) {
-    // accumulator columns 64 part .. + 63 are keys 64 (part & 1) .. + 63 of the tile for rows
-    // row0 + 128 (part >> 1) + (0..127)
-    const int rbase = row0 + 128 * (part >> 1) + (lane_row & ~31);   // first row of this warp
-    if (rbase >= r_end) return;                                      // the warp's rows are all padding
-    const int lane = lane_row & 31;
-    float* dst = out + static_cast<size_t>(rbase - P.row_begin) * P.c_stride +
-                 static_cast<size_t>(tile) * tc::kKeysPerTile + 64 * (part & 1);
+  auto epilogue = [&](int tile, int lane_row, int part, auto groups, float*, auto, uint64_t*) {
+    // accumulator lane = key lane_row of the tile, columns 64 part .. + 63 = rows row0 + 64 part + (0..63): for one
+    // row the 32 lanes of a warp hold 32 consecutive keys, so every store instruction writes one 128-byte line of
+    // that row and nothing has to be transposed
+    const int rb = row0 + 64 * part;   // the warp's first row (the same in every lane)
+    if (rb >= r_end) return;           // 64 padding rows
+    float* dst = out + static_cast<size_t>(rb - P.row_begin) * P.c_stride + static_cast<size_t>(tile) * tc::kKeysPerTile +
+                 lane_row;
+    const size_t stride = static_cast<size_t>(P.c_stride);
     groups([&](int g, float (&v)[32]) {
-      // through the scratch, sixteen columns at a time (16-byte pieces XOR-permuted by the row), so that the
-      // global stores are 64-byte runs of one row: 4 lanes per row, 8 rows per instruction
+      const int nv = r_end - (rb + 32 * g);   // rows of this group that exist (the same in every lane)
+      float* p = dst + static_cast<size_t>(32 * g) * stride;
+      if (nv >= 32) {
 #pragma unroll
-      for (int hsel = 0; hsel < 2; ++hsel) {
-        float4* mine = reinterpret_cast<float4*>(scratch + lane * 16);
+        for (int i = 0; i < 32; ++i) { *p = v[i] * sc; p += stride; }
+      } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int e = 16 * hsel + 4 * c;
-          mine[c ^ (lane & 3)] = make_float4(v[e] * sc, v[e + 1] * sc, v[e + 2] * sc, v[e + 3] * sc);
+        for (int i = 0; i < 32; ++i) {
+          if (i < nv) *p = v[i] * sc;
+          p += stride;
         }
-        __syncwarp();
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-          const int rr = it * 8 + (lane >> 2), c = lane & 3;
-          const float4 val = reinterpret_cast<const float4*>(scratch + rr * 16)[c ^ (rr & 3)];
-          if (rbase + rr < r_end)
-            *reinterpret_cast<float4*>(dst + static_cast<size_t>(rr) * P.c_stride + g * 32 + hsel * 16 + c * 4) = val;
-        }
-        __syncwarp();
       }
     });
   };
-  if (!tc::scores_cta<false>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue) && threadIdx.x == 0)
+  if (!tc::scores_cta<true>(tc_smem, q_row, keys, C, tile_begin, tile_end, epilogue) && threadIdx.x == 0)
     atomicCAS(&err[0], 0, HKV_ERR_TIMEOUT);
 }
 
